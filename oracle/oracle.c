@@ -1,0 +1,273 @@
+/*
+ * CPU oracle for the FreeCache denoising-step hot path of a diffusion language model.
+ *
+ * TEST INFRASTRUCTURE ONLY.  This file is the plain, slow, obviously-correct statement of
+ * what the hot path computes.  It shares no code, header, table or helper with the CUDA
+ * library, and the CUDA library never calls it.  Only the tests, the smoke check and the
+ * CPU-baseline leg of the benchmark may load it.
+ *
+ * Precision: floating-point inputs are fp32 (bf16 bit patterns widened exactly by the
+ * caller); every sum, dot product and exponential is carried in fp64 and the result is
+ * rounded once to fp32.  Integer / byte work is exact.
+ *
+ * Every function below is pinned by CPU tests to something other than itself (fp64 brute
+ * force over the full sequence, closed forms, a library SDPA, hand-worked examples,
+ * exhaustive enumeration); none is "parity unpinned".
+ *
+ * Notation follows the paper: M_t masked set (Eq. 1), z_t logits (Eq. 2), U_t selected set
+ * (Eq. 3), blocks B_1..B_N with frozen K/V (Sec. 3.2.1), tok_DLM / tok_AR and the masked
+ * index list M = [i_1..i_m] (Algorithm 1).
+ */
+#include <math.h>
+#include <stdint.h>
+#include <stdlib.h>
+#include <string.h>
+#ifdef _OPENMP
+#include <omp.h>
+#endif
+
+#define ORACLE_OK 0
+#define ORACLE_ERR_CAPACITY 1 /* bit: an append would run past the cache capacity      */
+#define ORACLE_ERR_INDEX 2    /* bit: a source or destination row index is out of range */
+
+int oracle_num_threads(void) {
+#ifdef _OPENMP
+  return omp_get_max_threads();
+#else
+  return 1;
+#endif
+}
+
+/*
+ * One attention step of one layer (Sec. 3.2.1, "Windowed Re-computation"; Table 1 rows
+ * QK^T and Attention Score x Value).
+ *
+ * For batch element b, query head h (KV head h / (Hq/Hkv)) and active row i < q_len[b]:
+ * the keys are the visible cached rows j < cache_len[b] (prompt and frozen blocks) followed
+ * by the freshly recomputed rows of the active window j' < q_len[b].  There is no causal
+ * mask (the model is bidirectional).  With s_j = scale * <q_i, k_j>:
+ *     out_i = sum_j softmax(s)_j * v_j,        lse_i = log sum_j exp(s_j).
+ * Rows i >= q_len[b] are defined as zero (lse = -inf).
+ *
+ * Layouts (row-major, innermost last):
+ *   cache_k, cache_v : [B][Hkv][Lcap][D]      q   : [B][Hq][q_cap][D]
+ *   k_new, v_new     : [B][Hkv][q_cap][D]     out : [B][Hq][q_cap][D]   lse : [B][Hq][q_cap]
+ *   cache_len, q_len : [B]  (q_len may be NULL: every row active)
+ * Rows of the cache at or beyond cache_len[b] are never read.
+ */
+int oracle_attn_step(int B, int Hq, int Hkv, int D, int Lcap, int q_cap,
+                     const float* cache_k, const float* cache_v, const int32_t* cache_len,
+                     const int32_t* q_len, const float* q, const float* k_new,
+                     const float* v_new, float scale, float* out, float* lse) {
+  if (Hkv <= 0 || Hq % Hkv != 0) return -1;
+  const int g = Hq / Hkv;
+#pragma omp parallel for collapse(2) schedule(dynamic, 1)
+  for (int b = 0; b < B; ++b) {
+    for (int h = 0; h < Hq; ++h) {
+      const int kvh = h / g;
+      const int Lc = cache_len[b];
+      const int Lq = q_len ? q_len[b] : q_cap;
+      const int L = Lc + Lq;
+      double* s = (double*)malloc(sizeof(double) * (size_t)(L > 0 ? L : 1));
+      double* acc = (double*)malloc(sizeof(double) * (size_t)D);
+      const float* Kc = cache_k + ((size_t)b * Hkv + kvh) * (size_t)Lcap * D;
+      const float* Vc = cache_v + ((size_t)b * Hkv + kvh) * (size_t)Lcap * D;
+      const float* Kn = k_new + ((size_t)b * Hkv + kvh) * (size_t)q_cap * D;
+      const float* Vn = v_new + ((size_t)b * Hkv + kvh) * (size_t)q_cap * D;
+      for (int i = 0; i < q_cap; ++i) {
+        float* o = out + (((size_t)b * Hq + h) * q_cap + i) * D;
+        float* l = lse + ((size_t)b * Hq + h) * q_cap + i;
+        if (i >= Lq) {
+          for (int d = 0; d < D; ++d) o[d] = 0.0f;
+          *l = -INFINITY;
+          continue;
+        }
+        const float* qi = q + (((size_t)b * Hq + h) * q_cap + i) * D;
+        double m = -INFINITY;
+        for (int j = 0; j < L; ++j) {
+          const float* kj = (j < Lc) ? Kc + (size_t)j * D : Kn + (size_t)(j - Lc) * D;
+          double dot = 0.0;
+          for (int d = 0; d < D; ++d) dot += (double)qi[d] * (double)kj[d];
+          s[j] = (double)scale * dot;
+          if (s[j] > m) m = s[j];
+        }
+        double denom = 0.0;
+        for (int d = 0; d < D; ++d) acc[d] = 0.0;
+        for (int j = 0; j < L; ++j) {
+          const float* vj = (j < Lc) ? Vc + (size_t)j * D : Vn + (size_t)(j - Lc) * D;
+          const double p = exp(s[j] - m);
+          denom += p;
+          for (int d = 0; d < D; ++d) acc[d] += p * (double)vj[d];
+        }
+        for (int d = 0; d < D; ++d) o[d] = (float)(acc[d] / denom);
+        *l = (float)(m + log(denom));
+      }
+      free(s);
+      free(acc);
+    }
+  }
+  return ORACLE_OK;
+}
+
+/*
+ * KV-cache commit / refresh (Sec. 3.2.1, "Initialization and Partitioning" saves K/V,
+ * "Progressive Caching" freezes them).  Pure data movement on 16-bit patterns.
+ *
+ * For every layer in [layer_begin, layer_end), batch element b, r < n[b], KV head and both
+ * tensors:   cache[layer][b][head][dst(b,r)][:] = new[layer - layer_begin][b][head][src(b,r)][:]
+ * with src(b,r) = src_idx ? src_idx[b][r] : r   and
+ *      dst(b,r) = dst_pos ? dst_pos[b][r] : cache_len[b] + r      (append),
+ * n[b] = n_rows ? n_rows[b] : n_max.  If advance_len != 0, cache_len[b] += n[b] afterwards.
+ *
+ * Layouts: cache_k/v [NL][B][Hkv][Lcap][D]; k_new/v_new [layer_end-layer_begin][B][Hkv][src_len][D];
+ *          src_idx, dst_pos [B][n_max]; n_rows, cache_len [B].
+ *
+ * Input errors (returned as a bit mask, other batch elements unaffected):
+ *   - n[b] outside [0, n_max], or an append / advance that would pass Lcap: nothing is
+ *     written for b and cache_len[b] is left alone (ORACLE_ERR_CAPACITY);
+ *   - a source index outside [0, src_len) or a destination outside [0, Lcap): that row is
+ *     skipped (ORACLE_ERR_INDEX).
+ */
+int oracle_kv_cache_commit(int NL, int B, int Hkv, int Lcap, int D, uint16_t* cache_k,
+                           uint16_t* cache_v, int32_t* cache_len, const uint16_t* k_new,
+                           const uint16_t* v_new, int src_len, const int32_t* src_idx,
+                           const int32_t* dst_pos, const int32_t* n_rows, int n_max,
+                           int advance_len, int layer_begin, int layer_end) {
+  int status = ORACLE_OK;
+  if (layer_begin < 0 || layer_end > NL || layer_begin > layer_end) return -1;
+  for (int b = 0; b < B; ++b) {
+    const int n = n_rows ? n_rows[b] : n_max;
+    const int len0 = cache_len[b];
+    if (n < 0 || n > n_max) { status |= ORACLE_ERR_CAPACITY; continue; }
+    if ((dst_pos == NULL || advance_len) && (len0 < 0 || (int64_t)len0 + n > Lcap)) {
+      status |= ORACLE_ERR_CAPACITY;
+      continue;
+    }
+    for (int r = 0; r < n; ++r) {
+      const int64_t src = src_idx ? src_idx[(size_t)b * n_max + r] : r;
+      const int64_t dst = dst_pos ? dst_pos[(size_t)b * n_max + r] : (int64_t)len0 + r;
+      if (src < 0 || src >= src_len || dst < 0 || dst >= Lcap) { status |= ORACLE_ERR_INDEX; continue; }
+      for (int layer = layer_begin; layer < layer_end; ++layer) {
+        for (int h = 0; h < Hkv; ++h) {
+          const size_t to = ((((size_t)layer * B + b) * Hkv + h) * (size_t)Lcap + (size_t)dst) * D;
+          const size_t from = ((((size_t)(layer - layer_begin) * B + b) * Hkv + h) * (size_t)src_len + (size_t)src) * D;
+          memcpy(cache_k + to, k_new + from, sizeof(uint16_t) * (size_t)D);
+          memcpy(cache_v + to, v_new + from, sizeof(uint16_t) * (size_t)D);
+        }
+      }
+    }
+    if (advance_len) cache_len[b] = len0 + n;
+  }
+  return status;
+}
+
+/*
+ * Confidence scoring and top-k unmasking (Eq. 2, Eq. 3 and M_{t-1} = M_t \ U_t).
+ *
+ * For each masked position (b, i) with logit row z over the vocabulary:
+ *     tok  = lowest v attaining max_v z_v        (argmax of the softmax = argmax of z),
+ *     conf = max softmax probability = 1 / sum_v exp(z_v - max z)   (fp64 sum, rounded to fp32).
+ * Unmasked positions get tok = -1, conf = -1.
+ * If k > 0: with k_eff = min(k, |M_t| in this batch element), U_t is the k_eff masked
+ * positions of largest conf (compared as fp32), ties to the lowest position; then
+ * tokens[pos] = tok[pos], masked[pos] = 0, sel_idx[b][0..n_sel) = U_t ascending (rest -1),
+ * n_sel[b] = k_eff.  If k == 0 ("propose only") nothing but tok and conf is written,
+ * and sel_idx / n_sel may be NULL.
+ *
+ * Layouts: logits [B][Lblk][V] fp32; masked uint8 [B][Lblk]; tokens, tok int32 [B][Lblk];
+ *          conf fp32 [B][Lblk]; sel_idx int32 [B][k]; n_sel int32 [B].
+ */
+int oracle_unmask_select(int B, int Lblk, int V, const float* logits, uint8_t* masked,
+                         int32_t* tokens, int k, int32_t* tok, float* conf, int32_t* sel_idx,
+                         int32_t* n_sel) {
+#pragma omp parallel for collapse(2) schedule(dynamic, 1)
+  for (int b = 0; b < B; ++b) {
+    for (int i = 0; i < Lblk; ++i) {
+      const size_t p = (size_t)b * Lblk + i;
+      if (!masked[p]) { tok[p] = -1; conf[p] = -1.0f; continue; }
+      const float* z = logits + p * (size_t)V;
+      int best = 0;
+      for (int v = 1; v < V; ++v)
+        if (z[v] > z[best]) best = v; /* strict: the lowest index wins a tie */
+      double sum = 0.0;
+      for (int v = 0; v < V; ++v) sum += exp((double)z[v] - (double)z[best]);
+      tok[p] = best;
+      conf[p] = (float)(1.0 / sum);
+    }
+  }
+  if (k <= 0) return ORACLE_OK;
+  for (int b = 0; b < B; ++b) {
+    uint8_t* mk = masked + (size_t)b * Lblk;
+    const float* cf = conf + (size_t)b * Lblk;
+    uint8_t* chosen = (uint8_t*)calloc((size_t)Lblk, 1);
+    int n = 0;
+    for (int round = 0; round < k; ++round) {
+      int best = -1;
+      for (int i = 0; i < Lblk; ++i) {
+        if (!mk[i] || chosen[i]) continue;
+        if (best < 0 || cf[i] > cf[best]) best = i; /* strict: lowest position wins a tie */
+      }
+      if (best < 0) break;
+      chosen[best] = 1;
+      ++n;
+    }
+    int w = 0;
+    for (int i = 0; i < Lblk; ++i) {
+      if (!chosen[i]) continue;
+      sel_idx[(size_t)b * k + w++] = i;
+      tokens[(size_t)b * Lblk + i] = tok[(size_t)b * Lblk + i];
+      mk[i] = 0;
+    }
+    for (; w < k; ++w) sel_idx[(size_t)b * k + w] = -1;
+    n_sel[b] = n;
+    free(chosen);
+  }
+  return ORACLE_OK;
+}
+
+/*
+ * Guided Diffusion accept rule (Sec. 3.2.2; Algorithm 1).
+ *
+ * Per batch element, let M = [i_1 < ... < i_m] be the masked positions.  k is the largest
+ * prefix length with tok_dlm[i_j] == tok_ar[i_j] for all j <= k.  If k > 0 positions
+ * i_1..i_k are unmasked with the DLM proposals; otherwise only i_1 is unmasked (with the
+ * DLM proposal, or with the AR token when fallback_source == 1).  m == 0 accepts nothing.
+ * Outputs: accept[b][i] in {0,1}; acc_idx[b][0..n_acc) ascending accepted positions (rest -1);
+ * tokens[accepted] written, masked[accepted] cleared.
+ *
+ * Layouts: tok_dlm, tok_ar, tokens, acc_idx int32 [B][Lblk]; masked, accept uint8 [B][Lblk];
+ *          n_acc int32 [B].
+ */
+int oracle_guided_accept(int B, int Lblk, const int32_t* tok_dlm, const int32_t* tok_ar,
+                         uint8_t* masked, int32_t* tokens, int fallback_source,
+                         uint8_t* accept, int32_t* acc_idx, int32_t* n_acc) {
+  for (int b = 0; b < B; ++b) {
+    const size_t o = (size_t)b * Lblk;
+    int n = 0, first = -1, still_agreeing = 1;
+    for (int i = 0; i < Lblk; ++i) { accept[o + i] = 0; acc_idx[o + i] = -1; }
+    for (int i = 0; i < Lblk; ++i) {
+      if (!masked[o + i]) continue;
+      if (first < 0) first = i;
+      if (!still_agreeing) continue;
+      if (tok_dlm[o + i] == tok_ar[o + i]) {
+        accept[o + i] = 1;
+        acc_idx[o + n++] = i;
+      } else {
+        still_agreeing = 0;
+      }
+    }
+    int fallback = 0;
+    if (n == 0 && first >= 0) { /* no agreement at i_1: accept it alone */
+      accept[o + first] = 1;
+      acc_idx[o + n++] = first;
+      fallback = 1;
+    }
+    for (int j = 0; j < n; ++j) {
+      const int i = acc_idx[o + j];
+      tokens[o + i] = (fallback && fallback_source == 1) ? tok_ar[o + i] : tok_dlm[o + i];
+      masked[o + i] = 0;
+    }
+    n_acc[b] = n;
+  }
+  return ORACLE_OK;
+}
