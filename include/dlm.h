@@ -1,0 +1,204 @@
+/*
+ * dlm.h — C-ABI of the FreeCache denoising-step library for NVIDIA B200 (sm_100a).
+ *
+ * The library implements the per-step hot path of a diffusion language model (DLM) served
+ * with FreeCache and Guided Diffusion:
+ *
+ *   dlm_freecache_attn_step  bidirectional GQA attention of the active window over
+ *                            [frozen cache rows ; freshly recomputed rows]   (Sec. 3.2.1)
+ *   dlm_kv_cache_commit      writes K/V rows into the device-resident cache  (Sec. 3.2.1)
+ *   dlm_unmask_select        confidence = max softmax probability, argmax token,
+ *                            top-k unmasking                                (Eq. 1-3)
+ *   dlm_guided_accept        longest agreeing prefix between the DLM proposals and an
+ *                            autoregressive guider's argmax                 (Algorithm 1)
+ *
+ * Conventions
+ *   - Every function returns an int: DLM_OK (0) or a negative DLM_ERR_* code.  When an
+ *     argument error is returned nothing has been launched.
+ *   - Pointers documented "device" are caller-owned device pointers on the context's GPU and
+ *     must stay valid until the enqueued work has finished.  The library never allocates,
+ *     frees or retains tensor memory; the only device memory it owns is a few hundred bytes
+ *     of status and ticket words inside the context.
+ *   - `stream` is a cudaStream_t passed as void* (NULL = the default stream).  All calls
+ *     only enqueue work; none synchronises except dlm_get_status.
+ *   - Data-dependent errors (an index out of range, an append beyond capacity, a bounded
+ *     device-side wait that expired) cannot be detected on the host without a round trip.
+ *     The kernels suppress the offending writes, record the first such error in the
+ *     context's device status word, and dlm_get_status reports it.
+ *   - All tensors are contiguous, row-major, innermost dimension last.  bf16 means the
+ *     16-bit brain-float bit pattern.
+ *   - There is no CPU fallback: on a machine without a usable sm_100 device dlm_create fails.
+ */
+#ifndef DLM_H_
+#define DLM_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+enum {
+  DLM_OK = 0,
+  DLM_ERR_NULL = -1,        /* a required pointer is NULL                                  */
+  DLM_ERR_SHAPE = -2,       /* a size is non-positive or inconsistent                       */
+  DLM_ERR_UNSUPPORTED = -3, /* valid but not implemented (head_dim, group size, ...)        */
+  DLM_ERR_CAPACITY = -4,    /* cache_len + rows would exceed the cache capacity             */
+  DLM_ERR_WORKSPACE = -5,   /* workspace NULL, misaligned or too small                      */
+  DLM_ERR_CUDA = -6,        /* a CUDA runtime / driver call failed                          */
+  DLM_ERR_TIMEOUT = -7,     /* a bounded device-side wait expired (kernel gave up cleanly)  */
+  DLM_ERR_INDEX = -8        /* a row index read from device memory is out of range          */
+};
+
+typedef struct dlm_ctx dlm_ctx;
+
+/* Creates a context bound to CUDA device `device` (must be compute capability 10.x).
+ * The context owns only its status / ticket words.  Not thread-safe: use one context per
+ * host thread or serialise calls.  Kernels enqueued through one context on different
+ * streams must not overlap in time (they share the context's ticket words). */
+int dlm_create(dlm_ctx** out, int device);
+int dlm_destroy(dlm_ctx* ctx);
+
+/* Synchronises `stream`, returns the first data-dependent error recorded by any kernel
+ * since the last call (DLM_OK if none) and clears it. */
+int dlm_get_status(dlm_ctx* ctx, void* stream);
+
+/* Static, human-readable text for a return code. */
+const char* dlm_strerror(int code);
+
+/* Number of kernels this context has launched so far (host-side counter). */
+int64_t dlm_launch_count(const dlm_ctx* ctx);
+
+/* View of a caller-owned KV cache (Sec. 3.2.1: K/V of the prompt and of frozen blocks).
+ *   k, v       device, bf16 [n_layers][batch][n_kv_heads][capacity][head_dim]
+ *   cache_len  device, int32 [batch]: rows [0, cache_len[b]) are visible to attention.
+ * Rows at or beyond cache_len[b] may hold anything (stale, staged, NaN) and never
+ * influence a result. */
+typedef struct {
+  void* k;
+  void* v;
+  int32_t* cache_len;
+  int32_t n_layers, batch, n_kv_heads, capacity, head_dim;
+} dlm_kv_cache;
+
+/*
+ * dlm_kv_cache_commit — cache fill, refresh and freeze (Sec. 3.2.1: the initial pass "saves"
+ * K/V for the whole sequence; a finished block's K/V are "frozen").
+ *
+ * For every layer in [layer_begin, layer_end), batch element b, r < n(b), KV head, and both
+ * tensors:   cache[layer][b][head][dst(b,r)][:] = new[layer-layer_begin][b][head][src(b,r)][:]
+ *   src(b,r) = src_idx ? src_idx[b*n_max + r] : r
+ *   dst(b,r) = dst_pos ? dst_pos[b*n_max + r] : cache_len[b] + r        (append)
+ *   n(b)     = n_rows  ? n_rows[b]            : n_max
+ * If advance_len != 0, cache_len[b] += n(b) once all rows of the call are written.
+ *
+ *   k_new, v_new  device, bf16 [layer_end-layer_begin][batch][n_kv_heads][src_len][head_dim]
+ *   src_idx       device, int32 [batch][n_max] or NULL
+ *   dst_pos       device, int32 [batch][n_max] or NULL; destinations within one batch element
+ *                 must be distinct (duplicates race; the result is then one of the sources)
+ *   n_rows        device, int32 [batch] or NULL
+ * Argument errors: NULL cache / tensors, src_len <= 0, n_max <= 0, bad layer range,
+ * head_dim * 2 bytes not a multiple of 16.
+ * Data-dependent: n(b) outside [0, n_max], or an append / advance with cache_len[b] + n(b) >
+ * capacity: nothing is written for b, status DLM_ERR_CAPACITY; an index outside [0, src_len) /
+ * [0, capacity): that row is skipped, status DLM_ERR_INDEX.
+ */
+int dlm_kv_cache_commit(dlm_ctx* ctx, const dlm_kv_cache* cache, const void* k_new,
+                        const void* v_new, int src_len, const int32_t* src_idx,
+                        const int32_t* dst_pos, const int32_t* n_rows, int n_max,
+                        int advance_len, int layer_begin, int layer_end, void* stream);
+
+/* Bytes of device scratch dlm_freecache_attn_step needs for `n_layers_in_call` layers,
+ * `n_q_heads` query heads and `q_cap` active rows on this cache (split-KV partial results).
+ * Returns 0 on invalid arguments. */
+size_t dlm_attn_workspace_bytes(const dlm_ctx* ctx, const dlm_kv_cache* cache,
+                                int n_layers_in_call, int n_q_heads, int q_cap);
+
+/*
+ * dlm_freecache_attn_step — attention of the active window (Sec. 3.2.1 "Windowed
+ * Re-computation"; Table 1 rows QK^T and Attention Score x Value; no causal mask).
+ *
+ * For each layer l in [layer_begin, layer_end), batch element b, query head h (KV head
+ * h / (n_q_heads / n_kv_heads)) and active row i < q_len(b):
+ *     keys/values = cache rows [0, cache_len[b]) of layer l, then fresh rows [0, q_len(b))
+ *     out[l][b][h][i][:] = sum_j softmax_j(scale * <q_i, k_j>) v_j      (fp32 accumulate)
+ *     lse[l][b][h][i]    = log sum_j exp(scale * <q_i, k_j>)            (natural log)
+ * Rows i >= q_len(b) get out = 0 and lse = -inf.  More than one layer per call is only
+ * meaningful when all layers' Q/K/V exist up front (a synthetic stack); a real model calls
+ * it once per layer.
+ *
+ *   q            device, bf16 [layers][batch][n_q_heads][q_cap][head_dim]
+ *   k_new, v_new device, bf16 [layers][batch][n_kv_heads][q_cap][head_dim]
+ *   q_len        device, int32 [batch] or NULL (= q_cap for all)
+ *   softmax_scale  <= 0 selects 1/sqrt(head_dim)
+ *   cache_len_hint host upper bound on max_b cache_len[b] used only to size the launch;
+ *                  <= 0 means "capacity".  A hint below the true length costs speed, not
+ *                  correctness.
+ *   out          device, bf16 [layers][batch][n_q_heads][q_cap][head_dim]
+ *   lse          device, fp32 [layers][batch][n_q_heads][q_cap] or NULL
+ *   workspace    device, 256-byte aligned, at least dlm_attn_workspace_bytes(...)
+ * Supported: head_dim in {64, 128}; n_q_heads a multiple of n_kv_heads;
+ * (n_q_heads / n_kv_heads) * q_cap <= 256; q_cap >= 1.  Otherwise DLM_ERR_UNSUPPORTED.
+ * Data-dependent: cache_len[b] outside [0, capacity] or q_len[b] outside [0, q_cap] is
+ * clamped and recorded as DLM_ERR_CAPACITY; an expired device wait as DLM_ERR_TIMEOUT.
+ */
+int dlm_freecache_attn_step(dlm_ctx* ctx, const dlm_kv_cache* cache, int layer_begin,
+                            int layer_end, const void* q, const void* k_new, const void* v_new,
+                            int n_q_heads, int q_cap, const int32_t* q_len, float softmax_scale,
+                            int cache_len_hint, void* out, float* lse, void* workspace,
+                            size_t workspace_bytes, void* stream);
+
+/* Bytes of device scratch dlm_unmask_select needs (per-row partial reductions). */
+size_t dlm_unmask_workspace_bytes(const dlm_ctx* ctx, int batch, int block_len, int vocab);
+
+/*
+ * dlm_unmask_select — confidence scoring and top-k unmasking (Eq. 2: one logit row per masked
+ * position; Eq. 3: fill with the argmax; M_{t-1} = M_t \ U_t).
+ *
+ * For each masked (b, i):  tok = lowest v attaining max_v z_v,  conf = 1 / sum_v exp(z_v - max z)
+ * (the maximum softmax probability).  Unmasked positions get tok = -1, conf = -1.
+ * If k > 0, per batch element: k_eff = min(k, number of masked positions); U = the k_eff masked
+ * positions of largest conf, ties to the lowest position; tokens[U] = tok[U]; masked[U] = 0;
+ * sel_idx[b][0..k_eff) = U ascending, remaining entries -1; n_sel[b] = k_eff.
+ * If k == 0 ("propose only") only tok and conf are written; sel_idx / n_sel may be NULL.
+ *
+ *   logits   device, fp32 [batch][block_len][vocab]; -inf allowed, NaN / +inf unspecified
+ *   masked   device, uint8 [batch][block_len], in/out (non-zero = masked)
+ *   tokens   device, int32 [batch][block_len], in/out
+ *   tok      device, int32 [batch][block_len], out
+ *   conf     device, fp32  [batch][block_len], out
+ *   sel_idx  device, int32 [batch][k], out;   n_sel device, int32 [batch], out
+ *   workspace device, 16-byte aligned, at least dlm_unmask_workspace_bytes(...)
+ * Supported: block_len <= 1024.
+ */
+int dlm_unmask_select(dlm_ctx* ctx, const float* logits, int batch, int block_len, int vocab,
+                      uint8_t* masked, int32_t* tokens, int k, int32_t* tok, float* conf,
+                      int32_t* sel_idx, int32_t* n_sel, void* workspace, size_t workspace_bytes,
+                      void* stream);
+
+/*
+ * dlm_guided_accept — Guided Diffusion accept rule (Sec. 3.2.2 and Algorithm 1).
+ *
+ * Per batch element, with M = [i_1 < ... < i_m] the masked positions: k = the largest prefix
+ * length such that tok_dlm[i_j] == tok_ar[i_j] for all j <= k.  Positions i_1..i_k are
+ * accepted; if k == 0 and m > 0, i_1 alone is accepted.  Accepted positions receive the DLM
+ * token (fallback_source == 1: the lone fallback position receives the AR token instead),
+ * and their mask is cleared.
+ *
+ *   tok_dlm, tok_ar device, int32 [batch][block_len]  (tok_ar[i] is the guider's prediction
+ *                   FOR position i)
+ *   masked, tokens  device, in/out as in dlm_unmask_select
+ *   accept          device, uint8 [batch][block_len], out (1 = accepted)
+ *   acc_idx         device, int32 [batch][block_len], out: accepted positions ascending, rest -1
+ *   n_acc           device, int32 [batch], out
+ * Supported: block_len <= 1024.
+ */
+int dlm_guided_accept(dlm_ctx* ctx, const int32_t* tok_dlm, const int32_t* tok_ar, int batch,
+                      int block_len, uint8_t* masked, int32_t* tokens, int fallback_source,
+                      uint8_t* accept, int32_t* acc_idx, int32_t* n_acc, void* stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* DLM_H_ */

@@ -1,0 +1,167 @@
+"""ctypes binding of libdlm.so: argument marshalling only.
+
+Every function has the name and the argument order of its C counterpart in include/dlm.h.
+Tensors are torch CUDA tensors (PyTorch is used for device memory and streams only); each
+call passes raw device pointers and the current CUDA stream.  There is no fallback: if the
+library is missing or a call fails, an exception is raised.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+
+import torch
+
+from . import build as _build
+
+DLM_OK = 0
+DLM_ERR_NULL, DLM_ERR_SHAPE, DLM_ERR_UNSUPPORTED, DLM_ERR_CAPACITY = -1, -2, -3, -4
+DLM_ERR_WORKSPACE, DLM_ERR_CUDA, DLM_ERR_TIMEOUT, DLM_ERR_INDEX = -5, -6, -7, -8
+
+
+class DlmError(RuntimeError):
+    def __init__(self, code, where):
+        self.code = code
+        super().__init__(f"{where}: {dlm_strerror(code)} ({code})")
+
+
+class dlm_kv_cache(ctypes.Structure):
+    _fields_ = [("k", ctypes.c_void_p), ("v", ctypes.c_void_p), ("cache_len", ctypes.c_void_p),
+                ("n_layers", ctypes.c_int32), ("batch", ctypes.c_int32), ("n_kv_heads", ctypes.c_int32),
+                ("capacity", ctypes.c_int32), ("head_dim", ctypes.c_int32)]
+
+
+_lib = None
+
+
+def lib() -> ctypes.CDLL:
+    """Loads libdlm.so (in-tree).  Raises if it has not been built."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    path = _build.LIB
+    if not os.path.exists(path):
+        raise ImportError(f"{path} is missing: run `python -m paper_2505_21467_b200.build` "
+                          "(there is no CPU or PyTorch fallback)")
+    L = ctypes.CDLL(path)
+    vp, i32, f32, sz = ctypes.c_void_p, ctypes.c_int, ctypes.c_float, ctypes.c_size_t
+    L.dlm_create.argtypes = [ctypes.POINTER(vp), i32]
+    L.dlm_destroy.argtypes = [vp]
+    L.dlm_get_status.argtypes = [vp, vp]
+    L.dlm_strerror.argtypes = [i32]
+    L.dlm_strerror.restype = ctypes.c_char_p
+    L.dlm_launch_count.argtypes = [vp]
+    L.dlm_launch_count.restype = ctypes.c_int64
+    L.dlm_kv_cache_commit.argtypes = [vp, ctypes.POINTER(dlm_kv_cache), vp, vp, i32, vp, vp, vp, i32, i32,
+                                      i32, i32, vp]
+    L.dlm_attn_workspace_bytes.argtypes = [vp, ctypes.POINTER(dlm_kv_cache), i32, i32, i32]
+    L.dlm_attn_workspace_bytes.restype = sz
+    L.dlm_freecache_attn_step.argtypes = [vp, ctypes.POINTER(dlm_kv_cache), i32, i32, vp, vp, vp, i32, i32,
+                                          vp, f32, i32, vp, vp, vp, sz, vp]
+    L.dlm_unmask_workspace_bytes.argtypes = [vp, i32, i32, i32]
+    L.dlm_unmask_workspace_bytes.restype = sz
+    L.dlm_unmask_select.argtypes = [vp, vp, i32, i32, i32, vp, vp, i32, vp, vp, vp, vp, vp, sz, vp]
+    L.dlm_guided_accept.argtypes = [vp, vp, vp, i32, i32, vp, vp, i32, vp, vp, vp, vp]
+    for name in ("dlm_create", "dlm_destroy", "dlm_get_status", "dlm_kv_cache_commit",
+                 "dlm_freecache_attn_step", "dlm_unmask_select", "dlm_guided_accept"):
+        getattr(L, name).restype = i32
+    _lib = L
+    return L
+
+
+def dlm_strerror(code: int) -> str:
+    return lib().dlm_strerror(int(code)).decode()
+
+
+def _check(code, where):
+    if code != DLM_OK:
+        raise DlmError(code, where)
+
+
+def _ptr(t, dtype=None):
+    if t is None:
+        return None
+    if not (isinstance(t, torch.Tensor) and t.is_cuda and t.is_contiguous()):
+        raise TypeError("expected a contiguous CUDA tensor")
+    if dtype is not None and t.dtype != dtype:
+        raise TypeError(f"expected dtype {dtype}, got {t.dtype}")
+    return ctypes.c_void_p(t.data_ptr())
+
+
+def _stream():
+    return ctypes.c_void_p(torch.cuda.current_stream().cuda_stream)
+
+
+def dlm_create(device: int = 0) -> ctypes.c_void_p:
+    ctx = ctypes.c_void_p()
+    _check(lib().dlm_create(ctypes.byref(ctx), int(device)), "dlm_create")
+    return ctx
+
+
+def dlm_destroy(ctx) -> None:
+    _check(lib().dlm_destroy(ctx), "dlm_destroy")
+
+
+def dlm_get_status(ctx) -> int:
+    """Synchronises the current stream; returns (and clears) the first device-side error code."""
+    return int(lib().dlm_get_status(ctx, _stream()))
+
+
+def dlm_launch_count(ctx) -> int:
+    return int(lib().dlm_launch_count(ctx))
+
+
+def make_kv_cache(k: torch.Tensor, v: torch.Tensor, cache_len: torch.Tensor) -> dlm_kv_cache:
+    """View of caller-owned tensors: k, v bf16 [NL,B,Hkv,Lcap,D]; cache_len int32 [B]."""
+    if k.dtype != torch.bfloat16 or k.shape != v.shape or k.dim() != 5:
+        raise TypeError("k and v must be bf16 tensors of the same 5-d shape")
+    NL, B, Hkv, Lcap, D = k.shape
+    if cache_len.shape != (B,):
+        raise TypeError("cache_len must have shape [batch]")
+    c = dlm_kv_cache(_ptr(k).value, _ptr(v).value, _ptr(cache_len, torch.int32).value, NL, B, Hkv, Lcap, D)
+    c._keepalive = (k, v, cache_len)
+    return c
+
+
+def dlm_kv_cache_commit(ctx, cache, k_new, v_new, src_len, src_idx, dst_pos, n_rows, n_max, advance_len,
+                        layer_begin, layer_end) -> None:
+    _check(lib().dlm_kv_cache_commit(
+        ctx, ctypes.byref(cache), _ptr(k_new, torch.bfloat16), _ptr(v_new, torch.bfloat16), int(src_len),
+        _ptr(src_idx, torch.int32), _ptr(dst_pos, torch.int32), _ptr(n_rows, torch.int32), int(n_max),
+        int(bool(advance_len)), int(layer_begin), int(layer_end), _stream()), "dlm_kv_cache_commit")
+
+
+def dlm_attn_workspace_bytes(ctx, cache, n_layers_in_call, n_q_heads, q_cap) -> int:
+    return int(lib().dlm_attn_workspace_bytes(ctx, ctypes.byref(cache), int(n_layers_in_call), int(n_q_heads),
+                                              int(q_cap)))
+
+
+def dlm_freecache_attn_step(ctx, cache, layer_begin, layer_end, q, k_new, v_new, n_q_heads, q_cap, q_len,
+                            softmax_scale, cache_len_hint, out, lse, workspace) -> None:
+    _check(lib().dlm_freecache_attn_step(
+        ctx, ctypes.byref(cache), int(layer_begin), int(layer_end), _ptr(q, torch.bfloat16),
+        _ptr(k_new, torch.bfloat16), _ptr(v_new, torch.bfloat16), int(n_q_heads), int(q_cap),
+        _ptr(q_len, torch.int32), float(softmax_scale), int(cache_len_hint), _ptr(out, torch.bfloat16),
+        _ptr(lse, torch.float32), _ptr(workspace), workspace.numel() * workspace.element_size(), _stream()),
+        "dlm_freecache_attn_step")
+
+
+def dlm_unmask_workspace_bytes(ctx, batch, block_len, vocab) -> int:
+    return int(lib().dlm_unmask_workspace_bytes(ctx, int(batch), int(block_len), int(vocab)))
+
+
+def dlm_unmask_select(ctx, logits, batch, block_len, vocab, masked, tokens, k, tok, conf, sel_idx, n_sel,
+                      workspace) -> None:
+    _check(lib().dlm_unmask_select(
+        ctx, _ptr(logits, torch.float32), int(batch), int(block_len), int(vocab), _ptr(masked, torch.uint8),
+        _ptr(tokens, torch.int32), int(k), _ptr(tok, torch.int32), _ptr(conf, torch.float32),
+        _ptr(sel_idx, torch.int32), _ptr(n_sel, torch.int32), _ptr(workspace),
+        workspace.numel() * workspace.element_size(), _stream()), "dlm_unmask_select")
+
+
+def dlm_guided_accept(ctx, tok_dlm, tok_ar, batch, block_len, masked, tokens, fallback_source, accept,
+                      acc_idx, n_acc) -> None:
+    _check(lib().dlm_guided_accept(
+        ctx, _ptr(tok_dlm, torch.int32), _ptr(tok_ar, torch.int32), int(batch), int(block_len),
+        _ptr(masked, torch.uint8), _ptr(tokens, torch.int32), int(fallback_source), _ptr(accept, torch.uint8),
+        _ptr(acc_idx, torch.int32), _ptr(n_acc, torch.int32), _stream()), "dlm_guided_accept")

@@ -1,0 +1,66 @@
+// Context management of the DLM FreeCache library: creation, status word, error text.
+#include <new>
+
+#include "common.cuh"
+
+extern "C" int dlm_create(dlm_ctx** out, int device) {
+  if (!out) return DLM_ERR_NULL;
+  *out = nullptr;
+  int count = 0;
+  if (cudaGetDeviceCount(&count) != cudaSuccess || device < 0 || device >= count) return DLM_ERR_CUDA;
+  cudaDeviceProp prop;
+  DLM_CUDA_TRY(cudaGetDeviceProperties(&prop, device));
+  if (prop.major != 10) return DLM_ERR_UNSUPPORTED;  // the kernels are sm_100a only
+  int prev = 0;
+  DLM_CUDA_TRY(cudaGetDevice(&prev));
+  DLM_CUDA_TRY(cudaSetDevice(device));
+  dlm_ctx* ctx = new (std::nothrow) dlm_ctx();
+  if (!ctx) return DLM_ERR_CUDA;
+  ctx->device = device;
+  ctx->num_sms = prop.multiProcessorCount;
+  ctx->launches = 0;
+  ctx->encode_tiled = nullptr;
+  if (cudaMalloc(&ctx->words, sizeof(dlm_device_words)) != cudaSuccess ||
+      cudaMemset(ctx->words, 0, sizeof(dlm_device_words)) != cudaSuccess) {
+    delete ctx;
+    cudaSetDevice(prev);
+    return DLM_ERR_CUDA;
+  }
+  cudaSetDevice(prev);
+  *out = ctx;
+  return DLM_OK;
+}
+
+extern "C" int dlm_destroy(dlm_ctx* ctx) {
+  if (!ctx) return DLM_ERR_NULL;
+  cudaFree(ctx->words);
+  delete ctx;
+  return DLM_OK;
+}
+
+extern "C" int dlm_get_status(dlm_ctx* ctx, void* stream) {
+  if (!ctx) return DLM_ERR_NULL;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  int code = 0;
+  DLM_CUDA_TRY(cudaMemcpyAsync(&code, &ctx->words->status, sizeof(int), cudaMemcpyDeviceToHost, s));
+  DLM_CUDA_TRY(cudaMemsetAsync(&ctx->words->status, 0, sizeof(int), s));
+  DLM_CUDA_TRY(cudaStreamSynchronize(s));
+  return code;
+}
+
+extern "C" int64_t dlm_launch_count(const dlm_ctx* ctx) { return ctx ? ctx->launches : 0; }
+
+extern "C" const char* dlm_strerror(int code) {
+  switch (code) {
+    case DLM_OK: return "ok";
+    case DLM_ERR_NULL: return "a required pointer is NULL";
+    case DLM_ERR_SHAPE: return "a size is non-positive or inconsistent";
+    case DLM_ERR_UNSUPPORTED: return "configuration not supported";
+    case DLM_ERR_CAPACITY: return "cache length or row count exceeds capacity";
+    case DLM_ERR_WORKSPACE: return "workspace missing, misaligned or too small";
+    case DLM_ERR_CUDA: return "a CUDA call failed";
+    case DLM_ERR_TIMEOUT: return "a bounded device-side wait expired";
+    case DLM_ERR_INDEX: return "a row index is out of range";
+    default: return "unknown error code";
+  }
+}

@@ -1,0 +1,71 @@
+// dlm_guided_accept: the Guided Diffusion accept rule (Sec. 3.2.2, Algorithm 1).
+//
+// Integer-only and tiny (one block of positions per batch element), so it is bound by launch
+// latency.  One warp per batch element walks the block 32 positions at a time; ballots give
+// the masked set, the first disagreement and the ascending output order without any sort.
+#include "common.cuh"
+
+namespace {
+
+__global__ void __launch_bounds__(32)
+guided_accept_kernel(const int32_t* __restrict__ tok_dlm, const int32_t* __restrict__ tok_ar, int block_len,
+                     uint8_t* __restrict__ masked, int32_t* __restrict__ tokens, int fallback_source,
+                     uint8_t* __restrict__ accept, int32_t* __restrict__ acc_idx, int32_t* __restrict__ n_acc) {
+  const int b = blockIdx.x;
+  const int lane = threadIdx.x;
+  const size_t o = (size_t)b * block_len;
+  const unsigned lt_mask = (1u << lane) - 1u;
+  int n = 0;             // accepted so far (warp-uniform)
+  int first_masked = -1; // i_1
+  bool open = true;      // still inside the agreeing prefix
+  for (int base = 0; base < block_len; base += 32) {
+    const int i = base + lane;
+    const bool in = i < block_len;
+    const bool m = in && masked[o + i] != 0;
+    const int td = in ? tok_dlm[o + i] : 0;
+    const bool agree = m && td == tok_ar[in ? o + i : o];
+    const unsigned mm = __ballot_sync(0xffffffffu, m);
+    const unsigned dis = __ballot_sync(0xffffffffu, m && !agree);
+    if (first_masked < 0 && mm) first_masked = base + __ffs(mm) - 1;
+    bool mine = false;
+    if (open) {
+      const unsigned below_first_dis = dis ? ((1u << (__ffs(dis) - 1)) - 1u) : 0xffffffffu;
+      const unsigned acc = mm & below_first_dis;
+      mine = (acc >> lane) & 1u;
+      if (mine) {
+        acc_idx[o + n + __popc(acc & lt_mask)] = i;
+        tokens[o + i] = td;
+        masked[o + i] = 0;
+      }
+      n += __popc(acc);
+      if (dis) open = false;
+    }
+    if (in) accept[o + i] = mine ? 1 : 0;
+  }
+  __syncwarp();
+  if (n == 0 && first_masked >= 0) {  // no agreement at i_1: accept it alone
+    if (lane == 0) {
+      const size_t q = o + first_masked;
+      accept[q] = 1;
+      acc_idx[o] = first_masked;
+      tokens[q] = fallback_source == 1 ? tok_ar[q] : tok_dlm[q];
+      masked[q] = 0;
+    }
+    n = 1;
+  }
+  for (int j = n + lane; j < block_len; j += 32) acc_idx[o + j] = -1;
+  if (lane == 0) n_acc[b] = n;
+}
+
+}  // namespace
+
+extern "C" int dlm_guided_accept(dlm_ctx* ctx, const int32_t* tok_dlm, const int32_t* tok_ar, int batch,
+                                 int block_len, uint8_t* masked, int32_t* tokens, int fallback_source,
+                                 uint8_t* accept, int32_t* acc_idx, int32_t* n_acc, void* stream) {
+  if (!ctx || !tok_dlm || !tok_ar || !masked || !tokens || !accept || !acc_idx || !n_acc) return DLM_ERR_NULL;
+  if (batch <= 0 || block_len <= 0) return DLM_ERR_SHAPE;
+  if (block_len > 1024 || (fallback_source != 0 && fallback_source != 1)) return DLM_ERR_UNSUPPORTED;
+  guided_accept_kernel<<<batch, 32, 0, static_cast<cudaStream_t>(stream)>>>(
+      tok_dlm, tok_ar, block_len, masked, tokens, fallback_source, accept, acc_idx, n_acc);
+  return dlm_launch_ok(ctx, 1);
+}

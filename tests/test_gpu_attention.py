@@ -1,0 +1,157 @@
+"""GPU parity of dlm_freecache_attn_step against the CPU oracle, through the C-ABI.
+Tolerance (fp32 oracle, unit-scale bf16 inputs, bf16 output): max |err| <= 2e-2, mean |err| <= 2e-3."""
+import numpy as np
+import pytest
+import torch
+
+import paper_2505_21467_b200 as dlm
+from workloads import get_config, make_attn_inputs, make_cache, seed_for
+from helpers import Dev, assert_attn_close, gpu_attn_step, oracle_attn_layers
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def dev():
+    return Dev()
+
+
+def _i32(a):
+    return torch.tensor(np.asarray(a), dtype=torch.int32, device="cuda")
+
+
+def _case(dev, oracle, NL, B, Hq, Hkv, D, Lcap, q_cap, cache_len, q_len=None, seed=1, layer_begin=0, nl=None,
+          scale=0.0, layers=None, hint=0, device="cpu"):
+    nl = NL - layer_begin if nl is None else nl
+    ck, cv = make_cache(NL, B, Hkv, Lcap, D, seed, device=device)
+    q, kn, vn = make_attn_inputs(nl, B, Hq, Hkv, q_cap, D, seed + 1, device=device)
+    cl = _i32(cache_len)
+    ql = None if q_len is None else _i32(q_len)
+    out, lse = gpu_attn_step(dev, ck.cuda(), cv.cuda(), cl, q.cuda(), kn.cuda(), vn.cuda(), ql, scale, layer_begin,
+                             layer_begin + nl, hint=hint)
+    assert dev.status() == 0
+    ref = oracle_attn_layers(oracle, ck, cv, cl, q, kn, vn, ql, scale if scale > 0 else None, layer_begin, layers)
+    errs = [assert_attn_close(out, lse, ref[lc], lc) for lc in ref]
+    return out, lse, errs
+
+
+def test_tiny_config_full(dev, oracle):
+    cfg = get_config(0)
+    _case(dev, oracle, cfg.n_layers, cfg.batch, cfg.n_q_heads, cfg.n_kv_heads, cfg.head_dim, cfg.capacity,
+          cfg.block_len, [cfg.prompt_len], seed=seed_for(0))
+
+
+@pytest.mark.parametrize("Hq,Hkv,D,Lcap,q_cap,cache_len,q_len", [
+    (28, 4, 128, 700, 32, [517, 640], None),            # Dream group of 7: two M tiles, several K tiles, ragged tail
+    (28, 4, 128, 700, 32, [517, 0], [32, 7]),           # ragged active rows, one empty cache
+    (8, 8, 128, 400, 64, [333, 128], [64, 64]),         # MHA (LLaDA-like), block 64
+    (4, 2, 64, 300, 32, [1, 299], [5, 32]),             # head_dim 64
+    (2, 1, 64, 200, 128, [130, 77], [128, 100]),        # 256 query rows per KV head, fresh part spans a full tile
+    (6, 2, 128, 260, 20, [256, 255], [20, 0]),          # q_cap not a multiple of 16; one element fully inactive
+    (3, 3, 128, 129, 1, [129, 128], None),              # a single active row
+])
+def test_shapes_and_ragged_lengths(dev, oracle, Hq, Hkv, D, Lcap, q_cap, cache_len, q_len):
+    out, lse, _ = _case(dev, oracle, 2, 2, Hq, Hkv, D, Lcap, q_cap, cache_len, q_len, seed=Hq * 100 + q_cap)
+    if q_len is not None:
+        for b, n in enumerate(q_len):
+            assert torch.all(out[:, b, :, n:] == 0)
+
+
+def test_layer_range_and_explicit_scale(dev, oracle):
+    _case(dev, oracle, 5, 1, 4, 2, 128, 300, 32, [290], seed=9, layer_begin=2, nl=2, scale=0.05)
+
+
+def test_poisoned_invisible_rows_do_not_leak(dev, oracle):
+    """Rows at or beyond cache_len / q_len may hold NaN: the result must not change (bit for bit)."""
+    NL, B, Hq, Hkv, D, Lcap, q_cap = 1, 2, 14, 2, 128, 520, 32
+    ck, cv = make_cache(NL, B, Hkv, Lcap, D, 31, device="cuda")
+    q, kn, vn = make_attn_inputs(NL, B, Hq, Hkv, q_cap, D, 32, device="cuda")
+    cl, ql = _i32([300, 5]), _i32([32, 9])
+    base, base_lse = gpu_attn_step(dev, ck, cv, cl, q, kn, vn, ql)
+    nan = float("nan")
+    ck[:, 0, :, 300:] = nan; cv[:, 0, :, 300:] = nan
+    ck[:, 1, :, 5:] = nan; cv[:, 1, :, 5:] = nan
+    kn[:, 1, :, 9:] = nan; vn[:, 1, :, 9:] = nan; q[:, 1, :, 9:] = nan
+    out, lse = gpu_attn_step(dev, ck, cv, cl, q, kn, vn, ql)
+    assert dev.status() == 0
+    assert torch.equal(out, base) and torch.equal(lse, base_lse)
+    assert torch.isfinite(out.float()).all()
+
+
+def test_deterministic(dev):
+    ck, cv = make_cache(2, 1, 4, 1100, 128, 41, device="cuda")
+    q, kn, vn = make_attn_inputs(2, 1, 28, 4, 32, 128, 42, device="cuda")
+    cl = _i32([1056])
+    a, al = gpu_attn_step(dev, ck, cv, cl, q, kn, vn)
+    b, bl = gpu_attn_step(dev, ck, cv, cl, q, kn, vn)
+    assert torch.equal(a, b) and torch.equal(al, bl)
+
+
+def test_argument_errors(dev):
+    ck, cv = make_cache(1, 1, 2, 64, 128, 1, device="cuda")
+    cl = _i32([10])
+    cache = dlm.make_kv_cache(ck, cv, cl)
+    ws = dev.workspace(1 << 20)
+
+    def call(Hq=4, q_cap=32, D=128, layer_end=1, ws_=ws):
+        q = torch.zeros(1, 1, Hq, q_cap, D, dtype=torch.bfloat16, device="cuda")
+        kn = torch.zeros(1, 1, 2, q_cap, D, dtype=torch.bfloat16, device="cuda")
+        dlm.dlm_freecache_attn_step(dev.ctx, cache, 0, layer_end, q, kn, kn, Hq, q_cap, None, 0.0, 0,
+                                    torch.empty_like(q), None, ws_)
+
+    before = dlm.dlm_launch_count(dev.ctx)
+    for kwargs, code in ((dict(Hq=3), dlm.DLM_ERR_UNSUPPORTED), (dict(Hq=4, q_cap=200), dlm.DLM_ERR_UNSUPPORTED),
+                         (dict(layer_end=2), dlm.DLM_ERR_SHAPE),
+                         (dict(ws_=ws[8:]), dlm.DLM_ERR_WORKSPACE)):
+        with pytest.raises(dlm.DlmError) as e:
+            call(**kwargs)
+        assert e.value.code == code, kwargs
+    assert dlm.dlm_launch_count(dev.ctx) == before
+    ck96, cv96 = make_cache(1, 1, 2, 64, 96, 1, device="cuda")
+    cache96 = dlm.make_kv_cache(ck96, cv96, cl)
+    q = torch.zeros(1, 1, 2, 8, 96, dtype=torch.bfloat16, device="cuda")
+    with pytest.raises(dlm.DlmError) as e:
+        dlm.dlm_freecache_attn_step(dev.ctx, cache96, 0, 1, q, q, q, 2, 8, None, 0.0, 0, torch.empty_like(q), None, ws)
+    assert e.value.code == dlm.DLM_ERR_UNSUPPORTED
+
+
+def test_out_of_range_lengths_are_clamped_and_reported(dev):
+    ck, cv = make_cache(1, 2, 2, 64, 128, 1, device="cuda")
+    q, kn, vn = make_attn_inputs(1, 2, 4, 2, 16, 128, 2, device="cuda")
+    out, _ = gpu_attn_step(dev, ck, cv, _i32([65, 10]), q, kn, vn)
+    assert dev.status() == dlm.DLM_ERR_CAPACITY
+    ref, _ = gpu_attn_step(dev, ck, cv, _i32([64, 10]), q, kn, vn)
+    assert dev.status() == 0 and torch.equal(out, ref)
+
+
+def test_dream7b_full_size_layer_batched_first_and_last_step(dev, oracle):
+    """The benchmark's launch: all 28 layers in one call at the Dream-7B shape, at the first step
+    (cache 1024) and the last (cache 1248); oracle on layers {0, 14, 27}, all heads and rows."""
+    cfg = get_config(1)
+    for cache_len in (cfg.prompt_len, cfg.capacity - cfg.block_len):
+        _case(dev, oracle, cfg.n_layers, cfg.batch, cfg.n_q_heads, cfg.n_kv_heads, cfg.head_dim, cfg.capacity,
+              cfg.block_len, [cache_len], seed=seed_for(1, cache_len), layers=[0, 14, 27], hint=cache_len,
+              device="cuda")
+
+
+def test_guided_shape_ragged_batch8(dev, oracle):
+    """Config 5's shape: batch 8 with ragged cache_len and q_len (accepted prefixes shrink the window)."""
+    cfg = get_config(4)
+    cache_len = [1024, 1031, 1056, 1100, 1247, 1279, 1088, 1150]
+    q_len = [32, 25, 32, 20, 1, 1, 32, 2]
+    _case(dev, oracle, 3, cfg.batch, cfg.n_q_heads, cfg.n_kv_heads, cfg.head_dim, cfg.capacity, cfg.block_len,
+          cache_len, q_len, seed=seed_for(4), layers=[0, 2])
+
+
+def test_longctx_shape_sampled_layers(dev, oracle):
+    """Config 4: 16384 cached rows, Dream heads; 4 of the 28 layers resident, oracle on two of them."""
+    cfg = get_config(3)
+    _case(dev, oracle, 4, cfg.batch, cfg.n_q_heads, cfg.n_kv_heads, cfg.head_dim, cfg.prompt_len + cfg.block_len,
+          cfg.block_len, [cfg.prompt_len], seed=seed_for(3), layers=[0, 3], device="cuda")
+
+
+def test_llada_shape_sampled(dev, oracle):
+    """Config 3's shape at full batch / heads / lengths, 2 layers resident; oracle on one layer."""
+    cfg = get_config(2)
+    _case(dev, oracle, 2, cfg.batch, cfg.n_q_heads, cfg.n_kv_heads, cfg.head_dim, cfg.capacity, cfg.block_len,
+          [2048, 2112, 2496, 2300], seed=seed_for(2), layers=[1], device="cuda")
