@@ -1,0 +1,355 @@
+#!/usr/bin/env python
+"""Benchmark of the FreeCache denoising step on B200.
+
+One "step" is one pass of the whole hot path for one denoising step of the Dream-7B-shaped
+workload: attention of the active block over [cache ; fresh rows] for all 28 layers (one
+layer-batched launch: all layers' synthetic Q/K/V exist up front), confidence scoring + top-4
+unmasking over vocab 152064, and the cache commit (4 staged rows, or the whole block when it
+completes).  Steps cycle through the 64-step generation schedule (8 blocks x 8 steps; cache
+1024 -> 1248 rows, 32 -> 4 masked positions).
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--config NAME]
+
+Prints one JSON line (rank 0).  `value` is denoise steps/s with inputs resident in HBM; `e2e`
+is the same with the step's inputs copied from pinned host memory and the result read back.
+L2 is flushed between timed steps (the cache of this workload is smaller than L2).
+With --impl reference the CPU oracle is timed on a bounded sample instead.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import numpy as np  # noqa: E402
+import torch  # noqa: E402
+
+from workloads import (get_config, make_attn_inputs, make_cache, make_kv_rows, make_logits,  # noqa: E402
+                       seed_for, widen, bf16_bits)
+
+METRIC = "denoise_steps_per_s"
+UNIT = "steps/s"
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        p = json.load(open(path))
+        return {"hbm_gbs": float(p["hbm_gbs"]), "bf16_tflops": float(p["bf16_tflops"]), "source": "measured"}
+    return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "source": "fallback"}
+
+
+class ClockSampler:
+    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+    Q = ("clocks.sm,clocks.max.sm,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+         "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index):
+        self.index, self.proc, self.lines = index, None, []
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.index), f"--query-gpu={self.Q}",
+                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                         stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except OSError:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.lines.append(line.strip())
+
+    def stop(self):
+        if not self.proc:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        self.thread.join(timeout=2)
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for line in self.lines:
+            f = [x.strip() for x in line.split(",")]
+            if len(f) < 6 or not f[0].isdigit():
+                continue
+            sm.append(int(f[0])); mx.append(int(f[1]))
+            for n, v in zip(names, f[2:6]):
+                if v.lower().startswith("active"):
+                    reasons.add(n)
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "samples": len(sm), "reasons": sorted(reasons)}
+
+
+class Schedule:
+    """The 64-step generation schedule of the top-k policy (host-side bookkeeping only)."""
+
+    def __init__(self, cfg):
+        self.cfg = cfg
+        self.n = cfg.n_blocks * cfg.steps_per_block
+
+    def at(self, t):
+        cfg = self.cfg
+        t %= self.n
+        block, s = divmod(t, cfg.steps_per_block)
+        return {"block": block, "step_in_block": s, "cache_len": cfg.prompt_len + block * cfg.block_len,
+                "n_masked": cfg.block_len - s * cfg.top_k, "last": s == cfg.steps_per_block - 1}
+
+
+def attn_bytes(cfg, cache_len):
+    """Algorithmic bytes of one layer-batched attention launch: K/V rows read once per KV head, Q read,
+    O written (bf16)."""
+    L = cache_len + cfg.block_len
+    kv = 2 * 2 * cfg.batch * cfg.n_kv_heads * L * cfg.head_dim
+    qo = 2 * 2 * cfg.batch * cfg.n_q_heads * cfg.block_len * cfg.head_dim
+    return cfg.n_layers * (kv + qo)
+
+
+def attn_flops(cfg, cache_len):
+    return cfg.n_layers * 4 * cfg.batch * cfg.n_q_heads * cfg.block_len * (cache_len + cfg.block_len) * cfg.head_dim
+
+
+class Workload:
+    """Device-resident state of one sequence batch plus the per-step launch sequence."""
+
+    N_POOL = 2   # distinct synthetic input sets cycled across steps
+
+    def __init__(self, cfg, cfg_index, device):
+        import paper_2505_21467_b200 as dlm
+        self.dlm, self.cfg, self.dev = dlm, cfg, device
+        self.ctx = dlm.dlm_create(device.index)
+        s = seed_for(cfg_index)
+        B, Lblk, V = cfg.batch, cfg.block_len, cfg.vocab
+        self.ck, self.cv = make_cache(cfg.n_layers, B, cfg.n_kv_heads, cfg.capacity, cfg.head_dim, s, device)
+        self.cache_len = torch.full((B,), cfg.prompt_len, dtype=torch.int32, device=device)
+        self.cache = dlm.make_kv_cache(self.ck, self.cv, self.cache_len)
+        self.pool = [make_attn_inputs(cfg.n_layers, B, cfg.n_q_heads, cfg.n_kv_heads, Lblk, cfg.head_dim, s + 1 + i,
+                                      device) for i in range(self.N_POOL)]
+        self.logits = [make_logits(B, Lblk, V, cfg.logit_sigma, s + 10 + i, device) for i in range(self.N_POOL)]
+        self.out = torch.empty_like(self.pool[0][0])
+        self.masked = torch.ones(B, Lblk, dtype=torch.uint8, device=device)
+        self.tokens = torch.full((B, Lblk), -1, dtype=torch.int32, device=device)
+        self.tok = torch.empty(B, Lblk, dtype=torch.int32, device=device)
+        self.conf = torch.empty(B, Lblk, dtype=torch.float32, device=device)
+        self.sel_idx = torch.empty(B, cfg.top_k, dtype=torch.int32, device=device)
+        self.n_sel = torch.empty(B, dtype=torch.int32, device=device)
+        self.attn_ws = torch.empty(max(dlm.dlm_attn_workspace_bytes(self.ctx, self.cache, cfg.n_layers, cfg.n_q_heads,
+                                                                    Lblk), 256), dtype=torch.uint8, device=device)
+        self.unmask_ws = torch.empty(max(dlm.dlm_unmask_workspace_bytes(self.ctx, B, Lblk, V), 256),
+                                     dtype=torch.uint8, device=device)
+        self.flush = torch.empty(512 << 20, dtype=torch.uint8, device=device)   # 4x the 126 MB L2
+        self.sched = Schedule(cfg)
+        self.t = 0
+
+    def reset_block_state(self, st):
+        """Puts the device state where step `t` of the schedule expects it (not timed)."""
+        self.cache_len.fill_(st["cache_len"])
+        self.masked.zero_()
+        self.masked[:, :st["n_masked"]] = 1
+
+    def launch_step(self, st, inputs=None, logits=None, attn_event=None):
+        """Enqueues one denoising step: attention (all layers), unmask, commit."""
+        dlm, cfg = self.dlm, self.cfg
+        q, kn, vn = inputs if inputs is not None else self.pool[self.t % self.N_POOL]
+        lg = logits if logits is not None else self.logits[self.t % self.N_POOL]
+        dlm.dlm_freecache_attn_step(self.ctx, self.cache, 0, cfg.n_layers, q, kn, vn, cfg.n_q_heads, cfg.block_len,
+                                    None, 0.0, st["cache_len"], self.out, None, self.attn_ws)
+        if attn_event is not None:
+            attn_event.record()
+        dlm.dlm_unmask_select(self.ctx, lg, cfg.batch, cfg.block_len, cfg.vocab, self.masked, self.tokens, cfg.top_k,
+                              self.tok, self.conf, self.sel_idx, self.n_sel, self.unmask_ws)
+        if st["last"]:      # block complete: freeze all of its rows and make them visible
+            dlm.dlm_kv_cache_commit(self.ctx, self.cache, kn, vn, cfg.block_len, None, None, dlm.DLM_DST_APPEND, None,
+                                    cfg.block_len, 1, 0, cfg.n_layers)
+        else:               # stage the rows unmasked in this step at their own slots
+            dlm.dlm_kv_cache_commit(self.ctx, self.cache, kn, vn, cfg.block_len, self.sel_idx, None,
+                                    dlm.DLM_DST_WINDOW, self.n_sel, cfg.top_k, 0, 0, cfg.n_layers)
+
+    def run(self, steps, timed, e2e=False, host=None):
+        """Runs `steps` steps; returns (total_ms, attn_ms, attn_bytes, attn_flops)."""
+        tot = attn = 0.0
+        nbytes = nflops = 0
+        for _ in range(steps):
+            st = self.sched.at(self.t)
+            if st["step_in_block"] == 0 or not timed:
+                self.reset_block_state(st)
+            self.flush.zero_()                      # evict L2 between timed steps
+            e0, e1, e2 = (torch.cuda.Event(enable_timing=True) for _ in range(3))
+            if e2e:
+                hq, hk, hv, hl, h_sel, h_n, h_tok = host
+                torch.cuda.synchronize()
+                t0 = time.perf_counter()
+                q, kn, vn = (x.to(self.dev, non_blocking=True) for x in (hq, hk, hv))
+                lg = hl.to(self.dev, non_blocking=True)
+                self.launch_step(st, (q, kn, vn), lg)
+                h_sel.copy_(self.sel_idx, non_blocking=True)
+                h_n.copy_(self.n_sel, non_blocking=True)
+                h_tok.copy_(self.tokens, non_blocking=True)
+                torch.cuda.synchronize()
+                tot += (time.perf_counter() - t0) * 1e3
+            else:
+                e0.record()
+                self.launch_step(st, attn_event=e1)
+                e2.record()
+                e2.synchronize()
+                tot += e0.elapsed_time(e2)
+                attn += e0.elapsed_time(e1)
+                nbytes += attn_bytes(self.cfg, st["cache_len"])
+                nflops += attn_flops(self.cfg, st["cache_len"])
+            self.t += 1
+        return tot, attn, nbytes, nflops
+
+
+def cpu_oracle_sample(cfg, cfg_index, n_layers_sample):
+    """Times the CPU oracle, as it stands, on a bounded sample of one denoising step: attention for
+    `n_layers_sample` of the layers at the first step's lengths, one unmask over the full block and one
+    4-row commit; extrapolates to a whole step."""
+    import oracle
+    s = seed_for(cfg_index)
+    B, Lblk = cfg.batch, cfg.block_len
+    ck, cv = make_cache(1, B, cfg.n_kv_heads, cfg.capacity, cfg.head_dim, s)
+    q, kn, vn = make_attn_inputs(1, B, cfg.n_q_heads, cfg.n_kv_heads, Lblk, cfg.head_dim, s + 1)
+    args = (widen(ck[0]), widen(cv[0]), np.full((B,), cfg.prompt_len, np.int32), widen(q[0]), widen(kn[0]), widen(vn[0]))
+    t0 = time.perf_counter()
+    for _ in range(n_layers_sample):
+        oracle.attn_step(*args)
+    t_attn = (time.perf_counter() - t0) / n_layers_sample
+    logits = make_logits(B, Lblk, cfg.vocab, cfg.logit_sigma, s + 10).numpy()
+    masked, tokens = np.ones((B, Lblk), np.uint8), np.zeros((B, Lblk), np.int32)
+    t0 = time.perf_counter()
+    _, _, sel, n = oracle.unmask_select(logits, masked, tokens, cfg.top_k)
+    t_unmask = time.perf_counter() - t0
+    cks, cvs = bf16_bits(ck), bf16_bits(cv)
+    knb, vnb = bf16_bits(kn), bf16_bits(vn)
+    t0 = time.perf_counter()
+    oracle.kv_cache_commit(cks, cvs, np.full((B,), cfg.prompt_len, np.int32), knb, vnb, sel, None, n, cfg.top_k, dst_mode=1)
+    t_commit = (time.perf_counter() - t0) * cfg.n_layers
+    step_s = cfg.n_layers * t_attn + t_unmask + t_commit
+    return {"value": 1.0 / step_s, "unit": UNIT, "cores": oracle.num_threads(), "kind": "oracle",
+            "sample": f"attention of {n_layers_sample} of {cfg.n_layers} layers at cache_len {cfg.prompt_len} "
+                      f"(x{cfg.n_layers}/{n_layers_sample}), one unmask over {Lblk}x{cfg.vocab} logits, one 4-row commit",
+            "seconds_per_step": step_s}
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=64)
+    ap.add_argument("--warmup", type=int, default=8)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--config", default="dream7b")
+    args = ap.parse_args()
+    cfg = get_config(args.config)
+    cfg_index = ["tiny", "dream7b", "llada8b", "longctx", "guided"].index(cfg.name)
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    config = {"workload": f"{cfg.name}: Dream-7B-shaped attention stack, batch {cfg.batch} per GPU, {cfg.n_layers} layers, "
+                          f"{cfg.n_q_heads}q/{cfg.n_kv_heads}kv heads x {cfg.head_dim}, prompt {cfg.prompt_len} + {cfg.n_blocks} blocks of "
+                          f"{cfg.block_len}, {cfg.steps_per_block} steps/block, vocab {cfg.vocab}, top-{cfg.top_k}",
+              "attention_launch": "layer-batched (all layers in one call; synthetic stack)",
+              "l2": "flushed between timed steps (512 MB write)", "parallelism": f"replicated x{world} (independent sequences)"}
+
+    if args.impl == "reference":
+        if rank != 0:
+            return
+        vals = []
+        for _ in range(args.warmup):
+            cpu_oracle_sample(cfg, cfg_index, 1)
+        for _ in range(args.steps):
+            vals.append(cpu_oracle_sample(cfg, cfg_index, 2))
+        sec = statistics.mean(v["seconds_per_step"] for v in vals)
+        base = dict(vals[-1]); base["value"] = 1.0 / sec
+        print(json.dumps({"impl": "reference", "metric": METRIC, "value": 1.0 / sec, "unit": UNIT, "n_gpus": args.gpus,
+                          "steps": args.steps, "warmup": args.warmup, "ms_per_step": sec * 1e3, "higher_is_better": True,
+                          "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic", "config": config,
+                          "cpu_baseline": base,
+                          "e2e": {"value": 1.0 / sec, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}))
+        return
+
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: there is no CPU fallback")
+    torch.cuda.set_device(local_rank)
+    device = torch.device("cuda", local_rank)
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=device)
+    from paper_2505_21467_b200 import build as _b
+    if rank == 0:
+        _b.build()
+    if world > 1:
+        dist.barrier()
+    wl = Workload(cfg, cfg_index, device)
+    dlm = wl.dlm
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    wl.run(max(args.warmup, 3), timed=False)
+    wl.t = 0
+    sampler = ClockSampler(local_rank)
+    barrier()
+    sampler.start()
+    launches0 = dlm.dlm_launch_count(wl.ctx)
+    tot_ms, attn_ms, nbytes, nflops = wl.run(args.steps, timed=True)
+    launches = dlm.dlm_launch_count(wl.ctx) - launches0
+    barrier()
+    clocks = sampler.stop()
+    status = dlm.dlm_get_status(wl.ctx)
+    if status != 0:
+        raise SystemExit(f"device status {status}: {dlm.dlm_strerror(status)}")
+
+    # end to end: the step's inputs come from pinned host memory, the result goes back
+    pin = lambda t: t.cpu().pin_memory()  # noqa: E731
+    q, kn, vn = wl.pool[0]
+    host = (pin(q), pin(kn), pin(vn), pin(wl.logits[0]), pin(wl.sel_idx), pin(wl.n_sel), pin(wl.tokens))
+    h2d = sum(x.numel() * x.element_size() for x in host[:4])
+    d2h = sum(x.numel() * x.element_size() for x in host[4:])
+    wl.t = 0
+    wl.run(3, timed=False, e2e=True, host=host)
+    wl.t = 0
+    e2e_steps = min(args.steps, 32)
+    e2e_ms, _, _, _ = wl.run(e2e_steps, timed=True, e2e=True, host=host)
+
+    times = torch.tensor([tot_ms, attn_ms, e2e_ms], dtype=torch.float64, device=device)
+    if world > 1:
+        dist.all_reduce(times, op=dist.ReduceOp.MAX)
+    tot_ms, attn_ms, e2e_ms = times.tolist()
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return
+    peaks = measured_peaks()
+    attn_gbs = nbytes / (attn_ms * 1e-3) / 1e9
+    line = {
+        "metric": METRIC, "value": world * args.steps / (tot_ms * 1e-3), "unit": UNIT, "n_gpus": world,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": tot_ms / args.steps, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic", "config": config,
+        "clocks": clocks, "gpu_launches": int(launches),
+        "e2e": {"value": world * e2e_steps / (e2e_ms * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d,
+                "d2h_bytes_per_step": d2h, "steps": e2e_steps},
+        "roofline": {"kernel": "attention step (all layers, one launch)", "bound": "hbm", "achieved": attn_gbs,
+                     "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": attn_gbs / peaks["hbm_gbs"],
+                     "peak_source": peaks["source"], "traffic": None,
+                     "attn_us_per_launch": attn_ms * 1e3 / args.steps,
+                     "attn_tflops": nflops / (attn_ms * 1e-3) / 1e12,
+                     "algorithmic_bytes_per_launch": nbytes / args.steps},
+        "cpu_baseline": cpu_oracle_sample(cfg, cfg_index, 4),
+    }
+    print(json.dumps(line))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

@@ -51,6 +51,8 @@ enum {
   DLM_ERR_INDEX = -8        /* a row index read from device memory is out of range          */
 };
 
+enum { DLM_DST_APPEND = 0, DLM_DST_WINDOW = 1 }; /* dlm_kv_cache_commit: where rows go when dst_pos is NULL */
+
 typedef struct dlm_ctx dlm_ctx;
 
 /* Creates a context bound to CUDA device `device` (must be compute capability 10.x).
@@ -89,7 +91,10 @@ typedef struct {
  * For every layer in [layer_begin, layer_end), batch element b, r < n(b), KV head, and both
  * tensors:   cache[layer][b][head][dst(b,r)][:] = new[layer-layer_begin][b][head][src(b,r)][:]
  *   src(b,r) = src_idx ? src_idx[b*n_max + r] : r
- *   dst(b,r) = dst_pos ? dst_pos[b*n_max + r] : cache_len[b] + r        (append)
+ *   dst(b,r) = dst_pos ? dst_pos[b*n_max + r]
+ *            : dst_mode == DLM_DST_WINDOW ? cache_len[b] + src(b,r)   (row p of the active window
+ *                                            is staged at its own slot behind the visible rows)
+ *            : cache_len[b] + r                                       (DLM_DST_APPEND)
  *   n(b)     = n_rows  ? n_rows[b]            : n_max
  * If advance_len != 0, cache_len[b] += n(b) once all rows of the call are written.
  *
@@ -100,13 +105,14 @@ typedef struct {
  *   n_rows        device, int32 [batch] or NULL
  * Argument errors: NULL cache / tensors, src_len <= 0, n_max <= 0, bad layer range,
  * head_dim * 2 bytes not a multiple of 16.
+ * dst_mode other than the two constants is DLM_ERR_SHAPE; it is ignored when dst_pos is given.
  * Data-dependent: n(b) outside [0, n_max], or an append / advance with cache_len[b] + n(b) >
  * capacity: nothing is written for b, status DLM_ERR_CAPACITY; an index outside [0, src_len) /
  * [0, capacity): that row is skipped, status DLM_ERR_INDEX.
  */
 int dlm_kv_cache_commit(dlm_ctx* ctx, const dlm_kv_cache* cache, const void* k_new,
                         const void* v_new, int src_len, const int32_t* src_idx,
-                        const int32_t* dst_pos, const int32_t* n_rows, int n_max,
+                        const int32_t* dst_pos, int dst_mode, const int32_t* n_rows, int n_max,
                         int advance_len, int layer_begin, int layer_end, void* stream);
 
 /* Bytes of device scratch dlm_freecache_attn_step needs for `n_layers_in_call` layers,

@@ -73,7 +73,7 @@ def attn_step(cache_k, cache_v, cache_len, q, k_new, v_new, q_len=None, scale=No
 
 
 def kv_cache_commit(cache_k, cache_v, cache_len, k_new, v_new, src_idx=None, dst_pos=None,
-                    n_rows=None, n_max=None, advance_len=False, layer_begin=0, layer_end=None):
+                    n_rows=None, n_max=None, advance_len=False, layer_begin=0, layer_end=None, dst_mode=0):
     """In-place commit on uint16 bit patterns.  cache [NL,B,Hkv,Lcap,D], new
     [layer_end-layer_begin,B,Hkv,src_len,D].  Returns the error bit mask."""
     NL, B, Hkv, Lcap, D = cache_k.shape
@@ -87,7 +87,7 @@ def kv_cache_commit(cache_k, cache_v, cache_len, k_new, v_new, src_idx=None, dst
     return int(_load().oracle_kv_cache_commit(
         NL, B, Hkv, Lcap, D, _p(cache_k, np.uint16), _p(cache_v, np.uint16),
         _p(cache_len, np.int32), _p(k_new, np.uint16), _p(v_new, np.uint16), src_len,
-        _p(src_idx, np.int32), _p(dst_pos, np.int32), _p(n_rows, np.int32), n_max,
+        _p(src_idx, np.int32), _p(dst_pos, np.int32), int(dst_mode), _p(n_rows, np.int32), n_max,
         int(bool(advance_len)), layer_begin, layer_end))
 
 

@@ -116,7 +116,10 @@ int oracle_attn_step(int B, int Hq, int Hkv, int D, int Lcap, int q_cap,
  * For every layer in [layer_begin, layer_end), batch element b, r < n[b], KV head and both
  * tensors:   cache[layer][b][head][dst(b,r)][:] = new[layer - layer_begin][b][head][src(b,r)][:]
  * with src(b,r) = src_idx ? src_idx[b][r] : r   and
- *      dst(b,r) = dst_pos ? dst_pos[b][r] : cache_len[b] + r      (append),
+ *      dst(b,r) = dst_pos ? dst_pos[b][r]
+ *               : dst_mode == 1 ? cache_len[b] + src(b,r)   (row p of the active window is staged
+ *                                                            at its own slot behind the visible rows)
+ *               : cache_len[b] + r                          (append),
  * n[b] = n_rows ? n_rows[b] : n_max.  If advance_len != 0, cache_len[b] += n[b] afterwards.
  *
  * Layouts: cache_k/v [NL][B][Hkv][Lcap][D]; k_new/v_new [layer_end-layer_begin][B][Hkv][src_len][D];
@@ -131,7 +134,7 @@ int oracle_attn_step(int B, int Hq, int Hkv, int D, int Lcap, int q_cap,
 int oracle_kv_cache_commit(int NL, int B, int Hkv, int Lcap, int D, uint16_t* cache_k,
                            uint16_t* cache_v, int32_t* cache_len, const uint16_t* k_new,
                            const uint16_t* v_new, int src_len, const int32_t* src_idx,
-                           const int32_t* dst_pos, const int32_t* n_rows, int n_max,
+                           const int32_t* dst_pos, int dst_mode, const int32_t* n_rows, int n_max,
                            int advance_len, int layer_begin, int layer_end) {
   int status = ORACLE_OK;
   if (layer_begin < 0 || layer_end > NL || layer_begin > layer_end) return -1;
@@ -139,13 +142,15 @@ int oracle_kv_cache_commit(int NL, int B, int Hkv, int Lcap, int D, uint16_t* ca
     const int n = n_rows ? n_rows[b] : n_max;
     const int len0 = cache_len[b];
     if (n < 0 || n > n_max) { status |= ORACLE_ERR_CAPACITY; continue; }
-    if ((dst_pos == NULL || advance_len) && (len0 < 0 || (int64_t)len0 + n > Lcap)) {
+    const int append = (dst_pos == NULL && dst_mode == 0);
+    if ((append || advance_len) && (len0 < 0 || (int64_t)len0 + n > Lcap)) {
       status |= ORACLE_ERR_CAPACITY;
       continue;
     }
     for (int r = 0; r < n; ++r) {
       const int64_t src = src_idx ? src_idx[(size_t)b * n_max + r] : r;
-      const int64_t dst = dst_pos ? dst_pos[(size_t)b * n_max + r] : (int64_t)len0 + r;
+      const int64_t dst = dst_pos ? dst_pos[(size_t)b * n_max + r]
+                                  : (dst_mode == 1 ? (int64_t)len0 + src : (int64_t)len0 + r);
       if (src < 0 || src >= src_len || dst < 0 || dst >= Lcap) { status |= ORACLE_ERR_INDEX; continue; }
       for (int layer = layer_begin; layer < layer_end; ++layer) {
         for (int h = 0; h < Hkv; ++h) {

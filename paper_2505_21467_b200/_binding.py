@@ -17,6 +17,7 @@ from . import build as _build
 DLM_OK = 0
 DLM_ERR_NULL, DLM_ERR_SHAPE, DLM_ERR_UNSUPPORTED, DLM_ERR_CAPACITY = -1, -2, -3, -4
 DLM_ERR_WORKSPACE, DLM_ERR_CUDA, DLM_ERR_TIMEOUT, DLM_ERR_INDEX = -5, -6, -7, -8
+DLM_DST_APPEND, DLM_DST_WINDOW = 0, 1
 
 
 class DlmError(RuntimeError):
@@ -52,7 +53,7 @@ def lib() -> ctypes.CDLL:
     L.dlm_strerror.restype = ctypes.c_char_p
     L.dlm_launch_count.argtypes = [vp]
     L.dlm_launch_count.restype = ctypes.c_int64
-    L.dlm_kv_cache_commit.argtypes = [vp, ctypes.POINTER(dlm_kv_cache), vp, vp, i32, vp, vp, vp, i32, i32,
+    L.dlm_kv_cache_commit.argtypes = [vp, ctypes.POINTER(dlm_kv_cache), vp, vp, i32, vp, vp, i32, vp, i32, i32,
                                       i32, i32, vp]
     L.dlm_attn_workspace_bytes.argtypes = [vp, ctypes.POINTER(dlm_kv_cache), i32, i32, i32]
     L.dlm_attn_workspace_bytes.restype = sz
@@ -123,11 +124,11 @@ def make_kv_cache(k: torch.Tensor, v: torch.Tensor, cache_len: torch.Tensor) -> 
     return c
 
 
-def dlm_kv_cache_commit(ctx, cache, k_new, v_new, src_len, src_idx, dst_pos, n_rows, n_max, advance_len,
+def dlm_kv_cache_commit(ctx, cache, k_new, v_new, src_len, src_idx, dst_pos, dst_mode, n_rows, n_max, advance_len,
                         layer_begin, layer_end) -> None:
     _check(lib().dlm_kv_cache_commit(
         ctx, ctypes.byref(cache), _ptr(k_new, torch.bfloat16), _ptr(v_new, torch.bfloat16), int(src_len),
-        _ptr(src_idx, torch.int32), _ptr(dst_pos, torch.int32), _ptr(n_rows, torch.int32), int(n_max),
+        _ptr(src_idx, torch.int32), _ptr(dst_pos, torch.int32), int(dst_mode), _ptr(n_rows, torch.int32), int(n_max),
         int(bool(advance_len)), int(layer_begin), int(layer_end), _stream()), "dlm_kv_cache_commit")
 
 

@@ -22,7 +22,7 @@ struct CommitParams {
   const int32_t* src_idx;
   const int32_t* dst_pos;
   const int32_t* n_rows;
-  int n_max, src_len, advance_len, layer_begin, n_layers_call;
+  int n_max, src_len, advance_len, layer_begin, n_layers_call, dst_mode;
   int batch, n_kv_heads, capacity;
   int vec_per_row;       // head_dim * 2 / 16
   int vec_shift;         // log2(vec_per_row) or -1
@@ -35,7 +35,8 @@ struct CommitParams {
 __device__ __forceinline__ int valid_rows(const CommitParams& p, int b, int len0) {
   const int n = p.n_rows ? p.n_rows[b] : p.n_max;
   if (n < 0 || n > p.n_max) return -1;
-  if ((p.dst_pos == nullptr || p.advance_len) && (len0 < 0 || (long long)len0 + n > p.capacity)) return -1;
+  const bool append = p.dst_pos == nullptr && p.dst_mode == DLM_DST_APPEND;
+  if ((append || p.advance_len) && (len0 < 0 || (long long)len0 + n > p.capacity)) return -1;
   return n;
 }
 
@@ -73,7 +74,8 @@ __global__ void __launch_bounds__(kThreads) kv_commit_kernel(const CommitParams 
       }
       if (r >= n) continue;
       const long long src = p.src_idx ? p.src_idx[(long long)b * p.n_max + r] : r;
-      const long long dst = p.dst_pos ? p.dst_pos[(long long)b * p.n_max + r] : (long long)len0 + r;
+      const long long dst = p.dst_pos ? p.dst_pos[(long long)b * p.n_max + r]
+                                      : (long long)len0 + (p.dst_mode == DLM_DST_WINDOW ? src : r);
       if (src < 0 || src >= p.src_len || dst < 0 || dst >= p.capacity) {
         if (vec == 0 && h == 0 && lc == 0) dlm_set_status(p.status, DLM_ERR_INDEX);
         continue;
@@ -116,11 +118,11 @@ __global__ void __launch_bounds__(kThreads) kv_commit_kernel(const CommitParams 
 
 extern "C" int dlm_kv_cache_commit(dlm_ctx* ctx, const dlm_kv_cache* cache, const void* k_new,
                                    const void* v_new, int src_len, const int32_t* src_idx,
-                                   const int32_t* dst_pos, const int32_t* n_rows, int n_max,
+                                   const int32_t* dst_pos, int dst_mode, const int32_t* n_rows, int n_max,
                                    int advance_len, int layer_begin, int layer_end, void* stream) {
   if (!ctx || !cache || !cache->k || !cache->v || !cache->cache_len || !k_new || !v_new) return DLM_ERR_NULL;
   if (cache->n_layers <= 0 || cache->batch <= 0 || cache->n_kv_heads <= 0 || cache->capacity <= 0 ||
-      cache->head_dim <= 0 || src_len <= 0 || n_max <= 0)
+      cache->head_dim <= 0 || src_len <= 0 || n_max <= 0 || (dst_mode != DLM_DST_APPEND && dst_mode != DLM_DST_WINDOW))
     return DLM_ERR_SHAPE;
   if (layer_begin < 0 || layer_end > cache->n_layers || layer_begin >= layer_end) return DLM_ERR_SHAPE;
   if ((cache->head_dim * 2) % 16 != 0) return DLM_ERR_UNSUPPORTED;
@@ -138,6 +140,7 @@ extern "C" int dlm_kv_cache_commit(dlm_ctx* ctx, const dlm_kv_cache* cache, cons
   p.n_max = n_max;
   p.src_len = src_len;
   p.advance_len = advance_len ? 1 : 0;
+  p.dst_mode = dst_mode;
   p.layer_begin = layer_begin;
   p.n_layers_call = layer_end - layer_begin;
   p.batch = cache->batch;

@@ -24,7 +24,7 @@ def _i32(a):
 
 
 def _run_commit(dev, oracle, ck, cv, cache_len, kn, vn, src_idx=None, dst_pos=None, n_rows=None, n_max=None,
-                advance=False, layer_begin=0, layer_end=None, expect_status=0):
+                advance=False, layer_begin=0, layer_end=None, expect_status=0, dst_mode=0):
     """ck.. are CPU bf16 tensors; runs both sides and compares every byte."""
     NL = ck.shape[0]
     layer_end = NL if layer_end is None else layer_end
@@ -38,10 +38,10 @@ def _run_commit(dev, oracle, ck, cv, cache_len, kn, vn, src_idx=None, dst_pos=No
                                 None if src_idx is None else np.asarray(src_idx, np.int32),
                                 None if dst_pos is None else np.asarray(dst_pos, np.int32),
                                 None if n_rows is None else np.asarray(n_rows, np.int32), n_max, advance,
-                                layer_begin, layer_end)
+                                layer_begin, layer_end, dst_mode)
     g_ck, g_cv, g_len = ck.cuda(), cv.cuda(), _i32(cache_len)
     cache = dlm.make_kv_cache(g_ck, g_cv, g_len)
-    dlm.dlm_kv_cache_commit(dev.ctx, cache, kn.cuda(), vn.cuda(), src_len, _i32(src_idx), _i32(dst_pos),
+    dlm.dlm_kv_cache_commit(dev.ctx, cache, kn.cuda(), vn.cuda(), src_len, _i32(src_idx), _i32(dst_pos), dst_mode,
                             _i32(n_rows), n_max, advance, layer_begin, layer_end)
     st = dev.status()
     np.testing.assert_array_equal(bf16_bits(g_ck), o_ck)
@@ -80,6 +80,11 @@ def test_commit_ragged_scatter_append_and_layer_range(dev, oracle, D):
     # append with a source gather, advancing the visible length
     _run_commit(dev, oracle, ck, cv, [10, 200, 0], kn, vn, src, None, [37, 20, 1], advance=True, layer_begin=2,
                 layer_end=5)
+    # window staging: row p of the fresh block lands at cache_len + p; the last slot may overflow
+    _run_commit(dev, oracle, ck, cv, [10, 231, 0], kn, vn, src, None, [37, 20, 1], dst_mode=1, layer_begin=0,
+                layer_end=3)
+    _run_commit(dev, oracle, ck, cv, [10, 240, 0], kn, vn, src, None, [37, 37, 1], dst_mode=1, layer_begin=0,
+                layer_end=3, expect_status=1)
     # plain contiguous append of every source row
     _run_commit(dev, oracle, ck, cv, [10, 231, 0], kn, vn, advance=True, layer_begin=0, layer_end=3)
 
@@ -101,12 +106,13 @@ def test_commit_argument_errors_launch_nothing(dev):
     kn = make_kv_rows((1, 1, 1, 4, 64), 2, device="cuda")
     before = dlm.dlm_launch_count(dev.ctx)
     for kwargs, code in ((dict(src_len=0), dlm.DLM_ERR_SHAPE), (dict(n_max=0), dlm.DLM_ERR_SHAPE),
-                         (dict(layer_end=2), dlm.DLM_ERR_SHAPE), (dict(layer_begin=1), dlm.DLM_ERR_SHAPE)):
-        a = dict(src_len=4, n_max=4, layer_begin=0, layer_end=1)
+                         (dict(layer_end=2), dlm.DLM_ERR_SHAPE), (dict(layer_begin=1), dlm.DLM_ERR_SHAPE),
+                         (dict(dst_mode=2), dlm.DLM_ERR_SHAPE)):
+        a = dict(src_len=4, n_max=4, layer_begin=0, layer_end=1, dst_mode=0)
         a.update(kwargs)
         with pytest.raises(dlm.DlmError) as e:
-            dlm.dlm_kv_cache_commit(dev.ctx, cache, kn, kn, a["src_len"], None, None, None, a["n_max"], 0,
-                                    a["layer_begin"], a["layer_end"])
+            dlm.dlm_kv_cache_commit(dev.ctx, cache, kn, kn, a["src_len"], None, None, a["dst_mode"], None,
+                                    a["n_max"], 0, a["layer_begin"], a["layer_end"])
         assert e.value.code == code
     assert dlm.dlm_launch_count(dev.ctx) == before
 
@@ -124,6 +130,7 @@ def test_commit_dream7b_prompt_refresh_and_block_freeze_full_size(dev, oracle):
     vn = make_kv_rows((cfg.n_layers, cfg.batch, cfg.n_kv_heads, cfg.block_len, cfg.head_dim), s + 4)
     sel = [[2, 11, 12, 31]]
     _run_commit(dev, oracle, ck, cv, [1024], kn, vn, sel, [[1024 + p for p in sel[0]]], [4])
+    _run_commit(dev, oracle, ck, cv, [1056], kn, vn, sel, None, [3], dst_mode=1)   # staged in the window
     _run_commit(dev, oracle, ck, cv, [1024], kn, vn, advance=True)            # whole block frozen
 
 
@@ -180,8 +187,9 @@ def test_unmask_ragged_vocab_and_ties(dev, oracle, V):
     logits[0, rows[1]] = logits[0, rows[0]]          # bit-identical rows: exact confidence tie
     if V > 8:
         logits[1, np.flatnonzero(masked0[1])[0], V // 2:] = -float("inf")
-        logits[2, :, V - 3] = logits[2].max() + 1.0  # shared maximum near the ragged tail
-        logits[2, :, 5] = logits[2, :, V - 3]        # duplicate maximum: lowest index wins
+        r2 = np.flatnonzero(masked0[2])[:2]
+        logits[2, r2, V - 3] = logits[2].max() + 1.0  # maximum near the ragged tail ...
+        logits[2, r2[0], 5] = logits[2, r2[0], V - 3]  # ... and a duplicate of it: lowest index wins
     _, conf, _, _ = oracle.unmask_select(logits.numpy(), masked0.copy(), np.zeros((B, Lblk), np.int32), 0)
     if V > 1 and topk_margin(conf, masked0, k) < 1e-4:
         pytest.skip("near-tie between distinct rows: several top-k sets are acceptable")

@@ -253,3 +253,24 @@ def test_guided_exhaustive_agreement_patterns(oracle, m):
         np.testing.assert_array_equal(acc_idx[b, :want], pos[:want])
         assert accept[b].sum() == want and masked[b].sum() == m - want
         np.testing.assert_array_equal(tokens[b, pos[:want]], dlm[b, pos[:want]])
+
+
+def test_commit_window_mode_stages_rows_at_their_own_slots(oracle):
+    """dst_mode 1: fresh row p goes to slot cache_len + p, whatever its place in the index list."""
+    ck, cv, kn, vn = _commit_case(500)
+    ck0 = ck.copy()
+    cache_len = np.array([5, 14], np.int32)
+    src_idx = np.array([[4, 1], [5, 0]], np.int32)
+    rc = oracle.kv_cache_commit(ck, cv, cache_len, kn, vn, src_idx, None, np.array([2, 2], np.int32), dst_mode=1)
+    assert rc == 0
+    np.testing.assert_array_equal(ck[:, 0, :, 9], kn[:, 0, :, 4])
+    np.testing.assert_array_equal(ck[:, 0, :, 6], kn[:, 0, :, 1])
+    np.testing.assert_array_equal(ck[:, 1, :, 19], kn[:, 1, :, 5])
+    np.testing.assert_array_equal(cv[:, 1, :, 14], vn[:, 1, :, 0])
+    ck[:, 0, :, [9, 6]] = ck0[:, 0, :, [9, 6]]
+    ck[:, 1, :, [19, 14]] = ck0[:, 1, :, [19, 14]]
+    np.testing.assert_array_equal(ck, ck0)
+    np.testing.assert_array_equal(cache_len, [5, 14])
+    cache_len = np.array([5, 15], np.int32)                     # 15 + 5 = 20 is past the last slot
+    assert oracle.kv_cache_commit(ck, cv, cache_len, kn, vn, src_idx, None, np.array([2, 2], np.int32),
+                                  dst_mode=1) == oracle.ERR_INDEX
