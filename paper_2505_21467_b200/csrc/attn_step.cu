@@ -371,7 +371,7 @@ attn_step_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
         }
         // every MMA issued by this thread has finished before TMEM is released
         tc_commit(bar_drain);
-        mbar_wait(bar_drain, 0, abort_ptr);
+        mbar_wait(bar_drain, 0, &never_flag);
       }
     } else {
       // ============================================================= softmax warpgroups
@@ -390,6 +390,11 @@ attn_step_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
         uint32_t gt = 0;
         bool ok = true;
         uint32_t v[32];
+        // the warp leaves a wait together, so the .sync.aligned TMEM instructions that follow
+        // always see a converged warp, also when a wait is given up
+        auto wait_warp = [&](uint32_t bar, uint32_t parity) {
+          return __all_sync(0xffffffffu, mbar_wait(bar, parity, abort_ptr)) != 0;
+        };
         while (ok && walk.next(g, n_cta)) {
           const int n = g.t_end - g.t_begin;
           const size_t qrow = (((size_t)g.lc_layer * p.batch + g.b) * p.n_q_heads + (size_t)g.kvh * p.group + h_local) *
@@ -412,7 +417,7 @@ attn_step_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
               // V rows in [valid, n16) would be multiplied by P = 0: clear them so that stale
               // NaN / Inf bit patterns cannot reach O.
               const uint32_t vs = gt % KS;
-              ok = mbar_wait(bar_v_full + 8 * vs, (gt / KS) & 1, abort_ptr);
+              ok = wait_warp(bar_v_full + 8 * vs, (gt / KS) & 1);
               if (!ok) break;
               const int per_row = G::kPanels * 8;
               for (int idx = tid; idx < (n16 - valid) * per_row; idx += 128) {
@@ -422,7 +427,7 @@ attn_step_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
               }
               fence_proxy_async_smem();
             }
-            ok = mbar_wait(bar_s_ready + 8 * mt, gt & 1, abort_ptr);
+            ok = wait_warp(bar_s_ready + 8 * mt, gt & 1);
             if (!ok) break;
             tc_fence_after_sync();
             // pass 1: row maximum over the valid keys of this tile
@@ -442,7 +447,7 @@ attn_step_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
             const float m_new = fmaxf(m_run, mx * p.scale_log2);
             if (it > 0 && __any_sync(0xffffffffu, m_new > m_run)) {
               // some row of this warp has a new maximum: rescale the warp's O rows in TMEM
-              ok = mbar_wait(bar_o_done + 8 * mt, (gt - 1) & 1, abort_ptr);
+              ok = wait_warp(bar_o_done + 8 * mt, (gt - 1) & 1);
               if (!ok) break;
               tc_fence_after_sync();
               const float alpha = ex2_approx(m_run - m_new);
@@ -483,7 +488,7 @@ attn_step_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
           }
           if (!ok) break;
           // ---- epilogue of the segment: O is complete once the last P V product has finished
-          ok = mbar_wait(bar_o_done + 8 * mt, (gt - 1) & 1, abort_ptr);
+          ok = wait_warp(bar_o_done + 8 * mt, (gt - 1) & 1);
           if (!ok) break;
           tc_fence_after_sync();
           const bool active = real_row && i_row < g.Lq;
