@@ -184,6 +184,34 @@ int dlm_unmask_select(dlm_ctx* ctx, const float* logits, int batch, int block_le
                       void* stream);
 
 /*
+ * dlm_unmask_select_static — dlm_unmask_select for callers that cannot allocate device memory.
+ * (The paper has no counterpart: this is a deployment variant of the call above, with the same
+ * arithmetic and the same results.)
+ *
+ * Some hosts of this library may not call cudaMalloc at all: code that runs under a fixed
+ * memory plan handed out by an outer runtime, plug-ins whose allocator belongs to another
+ * component, or processes started after the device's memory has been given away.  Such a
+ * caller can own neither a context (dlm_create allocates) nor a workspace.  This entry point
+ * needs neither: the per-row partial reductions live in a 1 MiB array that is part of the
+ * library's device image (every GPU that loads the library holds it until the process exits).
+ * It calls no allocating routine, takes no context and reports errors only by return code.
+ *
+ * Arguments and results are those of dlm_unmask_select (device pointers, same layouts), for
+ * the device that is current on the calling thread.
+ * Limit: batch * block_len * ceil(vocab / 4096) <= 65536, otherwise DLM_ERR_WORKSPACE and
+ * nothing is launched.
+ * The first call on each device looks up the array's device address (a driver query, made
+ * with that device current); make that first call before starting any stream capture.
+ * Every call on a device shares the one array and leaves its last contents in it.  Nothing
+ * in it has to start at zero (each call overwrites the entries it later reads), but two
+ * calls that may overlap on the GPU, from different streams or threads, race on it: order them.
+ * Not thread-safe for the first call on a device; serialise that one.
+ */
+int dlm_unmask_select_static(const float* logits, int batch, int block_len, int vocab,
+                             uint8_t* masked, int32_t* tokens, int k, int32_t* tok, float* conf,
+                             int32_t* sel_idx, int32_t* n_sel, void* stream);
+
+/*
  * dlm_guided_accept — Guided Diffusion accept rule (Sec. 3.2.2 and Algorithm 1).
  *
  * Per batch element, with M = [i_1 < ... < i_m] the masked positions: k = the largest prefix

@@ -62,9 +62,10 @@ def lib() -> ctypes.CDLL:
     L.dlm_unmask_workspace_bytes.argtypes = [vp, i32, i32, i32]
     L.dlm_unmask_workspace_bytes.restype = sz
     L.dlm_unmask_select.argtypes = [vp, vp, i32, i32, i32, vp, vp, i32, vp, vp, vp, vp, vp, sz, vp]
+    L.dlm_unmask_select_static.argtypes = [vp, i32, i32, i32, vp, vp, i32, vp, vp, vp, vp, vp]
     L.dlm_guided_accept.argtypes = [vp, vp, vp, i32, i32, vp, vp, i32, vp, vp, vp, vp]
     for name in ("dlm_create", "dlm_destroy", "dlm_get_status", "dlm_kv_cache_commit",
-                 "dlm_freecache_attn_step", "dlm_unmask_select", "dlm_guided_accept"):
+                 "dlm_freecache_attn_step", "dlm_unmask_select", "dlm_unmask_select_static", "dlm_guided_accept"):
         getattr(L, name).restype = i32
     _lib = L
     return L
@@ -158,6 +159,14 @@ def dlm_unmask_select(ctx, logits, batch, block_len, vocab, masked, tokens, k, t
         _ptr(tokens, torch.int32), int(k), _ptr(tok, torch.int32), _ptr(conf, torch.float32),
         _ptr(sel_idx, torch.int32), _ptr(n_sel, torch.int32), _ptr(workspace),
         workspace.numel() * workspace.element_size(), _stream()), "dlm_unmask_select")
+
+
+def dlm_unmask_select_static(logits, batch, block_len, vocab, masked, tokens, k, tok, conf, sel_idx, n_sel) -> None:
+    """dlm_unmask_select without a context or a workspace (scratch is a fixed array inside the library)."""
+    _check(lib().dlm_unmask_select_static(
+        _ptr(logits, torch.float32), int(batch), int(block_len), int(vocab), _ptr(masked, torch.uint8),
+        _ptr(tokens, torch.int32), int(k), _ptr(tok, torch.int32), _ptr(conf, torch.float32),
+        _ptr(sel_idx, torch.int32), _ptr(n_sel, torch.int32), _stream()), "dlm_unmask_select_static")
 
 
 def dlm_guided_accept(ctx, tok_dlm, tok_ar, batch, block_len, masked, tokens, fallback_source, accept,

@@ -200,3 +200,47 @@ extern "C" int dlm_unmask_select(dlm_ctx* ctx, const float* logits, int batch, i
                                                  sel_idx, n_sel);
   return dlm_launch_ok(ctx, 2);
 }
+
+// ---------------------------------------------------------------------------------------
+// dlm_unmask_select_static: the same two kernels with the per-row partial reductions kept in
+// a fixed device array that is part of the library image, for callers that cannot allocate
+// device memory at all.
+namespace {
+
+constexpr int kStaticTriples = 65536;  // 1 MiB: rows x chunks of one call may not exceed this
+static __device__ __align__(256) Triple g_static_partial[kStaticTriples];
+
+constexpr int kMaxDevices = 64;
+Triple* g_static_partial_addr[kMaxDevices];  // device address of the array, per device (0 = not looked up yet)
+
+}  // namespace
+
+extern "C" int dlm_unmask_select_static(const float* logits, int batch, int block_len, int vocab,
+                                        uint8_t* masked, int32_t* tokens, int k, int32_t* tok, float* conf,
+                                        int32_t* sel_idx, int32_t* n_sel, void* stream) {
+  if (!logits || !masked || !tok || !conf) return DLM_ERR_NULL;
+  if (k > 0 && (!tokens || !sel_idx || !n_sel)) return DLM_ERR_NULL;
+  if (batch <= 0 || block_len <= 0 || vocab <= 0 || k < 0) return DLM_ERR_SHAPE;
+  if (block_len > kMaxBlockLen || (long long)batch * block_len > 65535) return DLM_ERR_UNSUPPORTED;
+  if (((uintptr_t)logits & 3) != 0) return DLM_ERR_UNSUPPORTED;
+  const int n_chunks = (vocab + kChunk - 1) / kChunk;
+  if ((long long)batch * block_len * n_chunks > kStaticTriples) return DLM_ERR_WORKSPACE;
+  int device = -1;
+  DLM_CUDA_TRY(cudaGetDevice(&device));
+  if (device < 0 || device >= kMaxDevices) return DLM_ERR_UNSUPPORTED;
+  if (!g_static_partial_addr[device]) {
+    // In host code the array's name is only a handle; its address on the current device has to be
+    // asked for, once per device.
+    Triple* addr = nullptr;
+    if (cudaGetSymbolAddress(reinterpret_cast<void**>(&addr), g_static_partial) != cudaSuccess || !addr)
+      return DLM_ERR_CUDA;
+    g_static_partial_addr[device] = addr;
+  }
+  Triple* partial = g_static_partial_addr[device];
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  vocab_reduce_kernel<<<dim3(n_chunks, batch * block_len), kThreads, 0, s>>>(logits, masked, vocab, n_chunks, partial);
+  const int threads = ((block_len + 31) / 32) * 32;
+  unmask_select_kernel<<<batch, threads, 0, s>>>(partial, n_chunks, block_len, k, masked, tokens, tok, conf,
+                                                 sel_idx, n_sel);
+  return cudaGetLastError() == cudaSuccess ? DLM_OK : DLM_ERR_CUDA;
+}
