@@ -45,6 +45,11 @@ extern "C" int dlm_get_status(dlm_ctx* ctx, void* stream) {
   DLM_CUDA_TRY(cudaMemcpyAsync(&code, &ctx->words->status, sizeof(int), cudaMemcpyDeviceToHost, s));
   DLM_CUDA_TRY(cudaMemsetAsync(&ctx->words->status, 0, sizeof(int), s));
   DLM_CUDA_TRY(cudaStreamSynchronize(s));
+  if (code != 0) {
+    // a kernel that gave up may have left its ticket words half counted
+    DLM_CUDA_TRY(cudaMemsetAsync(ctx->words, 0, sizeof(dlm_device_words), s));
+    DLM_CUDA_TRY(cudaStreamSynchronize(s));
+  }
   return code;
 }
 

@@ -7,21 +7,23 @@
 // read from HBM once per KV head.  Keys are visited in tiles of 128 rows: first the visible
 // cache rows, then the fresh rows.
 //
-// Block = 10 warps, one block per SM (persistent):
+// Block = 12 warps (three warpgroups), one block per SM (persistent):
 //   warps 0-3   softmax of M tile 0 (thread = query row = TMEM lane)
 //   warps 4-7   softmax of M tile 1
 //   warp  8     TMA producer (one lane): Q once per segment, K and V tiles through two rings
-//   warp  9     tcgen05.mma issuer (one lane): S = Q K^T into TMEM, then O += P V with P read
-//               from TMEM (it overwrites S in place as packed bf16)
-// Online softmax in fp32 with base-2 exponentials; O stays in TMEM and is rescaled only when
-// a row maximum grows.
+//   warp  9/10  tcgen05.mma issuer of M tile 0 / 1 (one lane each): S = Q K^T into TMEM, then
+//               O += P V with P read from TMEM (it overwrites S in place as packed bf16)
+//   warp  11    idle (fills the third warpgroup, which hands most of its registers over)
+// Online softmax in fp32 with base-2 exponentials; a whole score row sits in registers between
+// the maximum and the exponentials; O stays in TMEM and is rescaled only when a row maximum has
+// grown by more than a threshold.
 //
 // Scheduling.  Every (unit, key tile) pair is one item of a global list; block c takes the
 // contiguous share [c*T/G, (c+1)*T/G) of it.  A share covers whole units (result written
 // directly) and at most two partial units (unnormalised O, running max and sum written to the
-// workspace; a second kernel merges the partials of a unit in a fixed order, so the result is
-// deterministic).  With many more units than SMs the split is not worth its traffic and units
-// are dealt round-robin instead.
+// workspace).  The block that finishes the last piece of a unit merges all its pieces, always
+// in block order, so the result is deterministic.  With many more units than SMs the split is
+// not worth its traffic and units are dealt round-robin instead.
 #include <cuda.h>
 #include <cuda_bf16.h>
 #include <math_constants.h>
@@ -33,11 +35,14 @@ namespace {
 
 using namespace sm100;
 
-constexpr int kThreads = 320;
+constexpr int kThreads = 384;          // 3 warpgroups: two of softmax warps, one with the producer and the MMA issuers
 constexpr int kTileKeys = 128;
 constexpr int kPanelBytes = 128 * 128;   // one 64-element-wide panel of a 128-row tile
 constexpr int kMaxBatch = 1024;
 constexpr int kTmemCols = 512;
+constexpr int kRegsSoftmax = 216;     // registers per thread of the softmax warpgroups after setmaxnreg.inc
+constexpr int kRegsOther = 72;        // ... of the producer / MMA warpgroup after setmaxnreg.dec
+constexpr int kMaxGrid = 256;          // blocks of the persistent grid (one per SM)
 
 template <int D>
 struct Geometry {
@@ -54,8 +59,8 @@ struct AttnParams {
   const int32_t* q_len;
   __nv_bfloat16* out;
   float* lse;
-  float* ws_o;    // [2 * grid][n_mt * 128][D]   partial unnormalised O
-  float* ws_ml;   // [2 * grid][n_mt * 128][2]   partial (running max in log2 units, running sum)
+  float* ws_o;    // [2 * grid][n_mt][D][128]    partial unnormalised O, column-major per M tile
+  float* ws_ml;   // [2 * grid][n_mt][128][2]    partial (running max in log2 units, running sum)
   int nl, layer_begin, batch, n_kv_heads, n_q_heads, group, capacity, q_cap;
   int rows;        // group * q_cap: query rows per unit
   int n_mt;        // M tiles per unit (1 or 2)
@@ -63,6 +68,7 @@ struct AttnParams {
   int whole_units; // 1: deal whole units round-robin, no partials
   float scale_log2;
   int* status;
+  unsigned int* tickets;   // one zero-initialised counter per unit: pieces finished
 };
 
 // Per-block scheduling tables (shared memory).
@@ -70,6 +76,7 @@ struct Sched {
   int prefix[kMaxBatch + 1];  // prefix[b] = tiles of batch elements < b; prefix[batch] = sum
   int lc[kMaxBatch];          // clamped cache_len
   int lq[kMaxBatch];          // clamped q_len
+  int share_lo[kMaxGrid + 1]; // split mode: block c owns items [share_lo[c], share_lo[c + 1])
 };
 
 struct Segment {
@@ -85,22 +92,20 @@ __device__ __forceinline__ int tiles_of(int Lc, int Lq, int fresh_box) {
 }
 
 // Walks the segments of block `cta`.  Identical in every role, so the roles agree on the
-// sequence without communicating.
+// sequence without communicating.  Item counts fit 32 bits (the host refuses larger launches).
 struct SegmentWalker {
   const AttnParams& p;
   const Sched& s;
-  long long pos, end, range_begin;
+  int pos, end, range_begin;
   int unit, n_units;
-  __device__ SegmentWalker(const AttnParams& p_, const Sched& s_, int cta, int n_cta) : p(p_), s(s_) {
-    const long long sum = s.prefix[p.batch];
-    const long long total = sum * p.nl * p.n_kv_heads;
+  __device__ SegmentWalker(const AttnParams& p_, const Sched& s_, int cta) : p(p_), s(s_) {
     n_units = p.nl * p.n_kv_heads * p.batch;
     if (p.whole_units) {
       unit = cta;
       pos = end = range_begin = 0;
     } else {
-      range_begin = pos = total * cta / n_cta;
-      end = total * (cta + 1) / n_cta;
+      range_begin = pos = s.share_lo[cta];
+      end = s.share_lo[cta + 1];
       unit = 0;
     }
   }
@@ -122,12 +127,12 @@ struct SegmentWalker {
       return true;
     }
     if (pos >= end) return false;
-    const long long sum = s.prefix[p.batch];
-    const int grp = (int)(pos / sum);
-    const int rem = (int)(pos - (long long)grp * sum);
+    const int sum = s.prefix[p.batch];
+    const int grp = pos / sum;
+    const int rem = pos - grp * sum;
     int b = 0;
     while (s.prefix[b + 1] <= rem) ++b;   // batch is small; units with zero tiles are skipped
-    const long long unit_start = (long long)grp * sum + s.prefix[b];
+    const int unit_start = grp * sum + s.prefix[b];
     g.b = b;
     g.lc_layer = grp / p.n_kv_heads;
     g.kvh = grp % p.n_kv_heads;
@@ -135,9 +140,9 @@ struct SegmentWalker {
     g.Lq = s.lq[b];
     g.T = s.prefix[b + 1] - s.prefix[b];
     g.n_ct = (g.Lc + kTileKeys - 1) / kTileKeys;
-    g.t_begin = (int)(pos - unit_start);
-    const long long room = end - unit_start;
-    g.t_end = room < g.T ? (int)room : g.T;
+    g.t_begin = pos - unit_start;
+    const int room = end - unit_start;
+    g.t_end = room < g.T ? room : g.T;
     const bool whole = g.t_begin == 0 && g.t_end == g.T;
     g.slot = whole ? -1 : (pos == range_begin ? 2 * (int)blockIdx.x : 2 * (int)blockIdx.x + 1);
     pos = unit_start + g.t_end;
@@ -149,6 +154,164 @@ struct SegmentWalker {
 __device__ __forceinline__ int tile_valid(const Segment& g, int t, int fresh_box) {
   if (t < g.n_ct) return min(kTileKeys, g.Lc - t * kTileKeys);
   return min(fresh_box, g.Lq - (t - g.n_ct) * fresh_box);
+}
+
+// The blocks whose shares overlap the unit of segment g (this block is one of them), and where
+// each of them left its partial result.
+struct UnitPieces {
+  const Sched& s;
+  int u0, u1, c_first, c_last;
+  __device__ UnitPieces(const AttnParams& p, const Sched& s_, const Segment& g, int cta) : s(s_) {
+    const int sum = s.prefix[p.batch];
+    u0 = (g.lc_layer * p.n_kv_heads + g.kvh) * sum + s.prefix[g.b];
+    u1 = u0 + g.T;
+    c_first = c_last = cta;
+    while (s.share_lo[c_first] > u0) --c_first;
+    while (s.share_lo[c_last + 1] < u1) ++c_last;
+  }
+  // slot of the piece computed by block c (c_first <= c <= c_last): the block's first segment
+  // if the piece starts where the block's share starts, else its second one
+  __device__ __forceinline__ int slot_of(int c) const { return s.share_lo[c] >= u0 ? 2 * c : 2 * c + 1; }
+};
+
+// Softmax of one key tile for the query row held by this thread (S row in TMEM -> P row in TMEM).
+// O is rescaled only when the running maximum has grown by more than kRescaleThreshold (log2
+// units): until then P is formed against the older, smaller maximum and may reach
+// 2^kRescaleThreshold, which bf16 and the fp32 accumulators hold just as well; the final division
+// by the row sum, taken against the same maximum, cancels it.
+constexpr float kRescaleThreshold = 8.0f;
+
+// With two M tiles the exponentials of the two softmax groups take turns on the SFU: group 1 starts
+// those of a tile when group 0 has finished its own, and group 0 starts the next tile's when
+// group 1 is done.  Left alone the two groups drift into lockstep, and then the SFU and the
+// tensor pipe idle in turn; alternating, one group's exponentials run under the other's MMAs.
+struct ExpTurn {
+  uint32_t wait_bar;      // 0: nothing to wait for
+  uint32_t wait_parity;
+  uint32_t arrive_bar;    // 0: nobody to tell
+  volatile int* abort_ptr;
+  __device__ __forceinline__ bool begin() const {
+    if (wait_bar == 0) return true;
+    return __all_sync(0xffffffffu, mbar_wait(wait_bar, wait_parity, abort_ptr)) != 0;
+  }
+  __device__ __forceinline__ void end() const {
+    if (arrive_bar != 0) mbar_arrive(arrive_bar);
+  }
+};
+
+// Rare path shared by both tile kinds: some row of the warp outgrew its maximum by more than the
+// threshold, so the warp's O rows in TMEM are rescaled (rows that did not grow keep factor 1).
+// The P V product of the previous tile has finished by then: its issuer commits the barrier that
+// announced this tile's scores only after that product.
+template <int D>
+__device__ __noinline__ void rescale_o(uint32_t t_o, bool grow, float m_new, float& m_used, float& l_run) {
+  const float alpha = grow ? ex2_approx(m_used - m_new) : 1.0f;
+  uint32_t v[32];
+#pragma unroll 1
+  for (int c = 0; c < D / 32; ++c) {
+    tmem_ld32(t_o + c * 32, v);
+    tmem_ld_wait();
+#pragma unroll
+    for (int j = 0; j < 32; ++j) v[j] = __float_as_uint(__uint_as_float(v[j]) * alpha);
+    tmem_st32(t_o + c * 32, v);
+  }
+  l_run *= alpha;
+  if (grow) m_used = m_new;
+}
+
+// Full tile (128 valid keys): the whole score row sits in registers between the maximum and the
+// exponentials, so TMEM is read once and with a single wait.
+template <int D>
+__device__ __forceinline__ bool softmax_tile_full(uint32_t t_s, uint32_t t_o, bool first, float scale_log2,
+                                                  float& m_used, float& l_run, const ExpTurn& turn) {
+  uint32_t s[128];
+#pragma unroll
+  for (int c = 0; c < 4; ++c) tmem_ld32(t_s + c * 32, s + 32 * c);
+  tmem_ld_wait();
+  float mx[8];   // independent chains: the maximum is latency-bound otherwise
+#pragma unroll
+  for (int c = 0; c < 8; ++c) mx[c] = __uint_as_float(s[c]);
+#pragma unroll
+  for (int j = 8; j < 128; j += 8) {
+#pragma unroll
+    for (int c = 0; c < 8; ++c) mx[c] = fmaxf(mx[c], __uint_as_float(s[j + c]));
+  }
+  const float m_new =
+      fmaxf(fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3])), fmaxf(fmaxf(mx[4], mx[5]), fmaxf(mx[6], mx[7]))) * scale_log2;
+  if (first) {
+    m_used = m_new;
+    l_run = 0.f;
+  } else {
+    const bool grow = m_new > m_used + kRescaleThreshold;
+    if (__any_sync(0xffffffffu, grow)) rescale_o<D>(t_o, grow, m_new, m_used, l_run);
+  }
+  if (!turn.begin()) return false;
+  float l0 = 0.f, l1 = 0.f;
+#pragma unroll
+  for (int c = 0; c < 4; ++c) {
+    uint32_t pk[16];
+#pragma unroll
+    for (int j = 0; j < 16; ++j) {
+      const float p0 = ex2_approx(fmaf(__uint_as_float(s[32 * c + 2 * j]), scale_log2, -m_used));
+      const float p1 = ex2_approx(fmaf(__uint_as_float(s[32 * c + 2 * j + 1]), scale_log2, -m_used));
+      l0 += p0;
+      l1 += p1;
+      const __nv_bfloat162 h = __floats2bfloat162_rn(p0, p1);
+      pk[j] = *reinterpret_cast<const uint32_t*>(&h);
+    }
+    if (c == 3) turn.end();
+    tmem_st16(t_s + c * 16, pk);
+  }
+  l_run += l0 + l1;
+  tmem_st_wait();
+  return true;
+}
+
+// Ragged tile (fewer than 128 valid keys: the end of the cache rows, or the fresh rows): 32 columns
+// at a time, keys at or beyond `valid` masked out.
+template <int D>
+__device__ __noinline__ bool softmax_tile_ragged(uint32_t t_s, uint32_t t_o, int valid, bool first, float scale_log2,
+                                                 float& m_used, float& l_run, const ExpTurn& turn) {
+  const int n_chunks = (valid + 31) >> 5;
+  uint32_t v[32];
+  float mx = -CUDART_INF_F;
+  for (int c = 0; c < n_chunks; ++c) {
+    tmem_ld32(t_s + c * 32, v);
+    tmem_ld_wait();
+#pragma unroll
+    for (int j = 0; j < 32; ++j)
+      if (c * 32 + j < valid) mx = fmaxf(mx, __uint_as_float(v[j]));
+  }
+  const float m_new = mx * scale_log2;
+  if (first) {
+    m_used = m_new;
+    l_run = 0.f;
+  } else {
+    const bool grow = m_new > m_used + kRescaleThreshold;
+    if (__any_sync(0xffffffffu, grow)) rescale_o<D>(t_o, grow, m_new, m_used, l_run);
+  }
+  if (!turn.begin()) return false;
+  float l_add = 0.f;
+  for (int c = 0; c < n_chunks; ++c) {
+    tmem_ld32(t_s + c * 32, v);
+    tmem_ld_wait();
+    uint32_t pk[16];
+#pragma unroll
+    for (int j = 0; j < 16; ++j) {
+      float p0 = ex2_approx(fmaf(__uint_as_float(v[2 * j]), scale_log2, -m_used));
+      float p1 = ex2_approx(fmaf(__uint_as_float(v[2 * j + 1]), scale_log2, -m_used));
+      if (c * 32 + 2 * j >= valid) p0 = 0.f;
+      if (c * 32 + 2 * j + 1 >= valid) p1 = 0.f;
+      l_add += p0 + p1;
+      const __nv_bfloat162 h = __floats2bfloat162_rn(p0, p1);
+      pk[j] = *reinterpret_cast<const uint32_t*>(&h);
+    }
+    tmem_st16(t_s + c * 16, pk);
+  }
+  turn.end();
+  l_run += l_add;
+  tmem_st_wait();
+  return true;
 }
 
 template <int D>
@@ -163,24 +326,29 @@ attn_step_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
   __shared__ int abort_flag;
   __shared__ int never_flag;   // stays 0: for waits that must not be cut short by an abort
   __shared__ uint32_t tmem_slot;
+  __shared__ int merge_is_last;
+  __shared__ int merge_slot[kMaxGrid];
 
   const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
   const uint32_t sm_q = smem_base;                               // [2][kTileBytes]
   const uint32_t sm_k = sm_q + 2 * G::kTileBytes;                // [KS][kTileBytes]
   const uint32_t sm_v = sm_k + KS * G::kTileBytes;               // [KS][kTileBytes]
   const uint32_t sm_bar = sm_v + KS * G::kTileBytes;             // barriers, 8 bytes each
-  const uint32_t bar_q_full = sm_bar, bar_q_empty = sm_bar + 8, bar_drain = sm_bar + 16;
+  const uint32_t bar_q_full = sm_bar, bar_q_empty = sm_bar + 8, bar_drain = sm_bar + 16;   // drain: [2]
   const uint32_t bar_k_full = sm_bar + 32, bar_k_empty = bar_k_full + 8 * KS;
   const uint32_t bar_v_full = bar_k_empty + 8 * KS, bar_v_empty = bar_v_full + 8 * KS;
   const uint32_t bar_s_ready = bar_v_empty + 8 * KS;             // [2]
   const uint32_t bar_p_ready = bar_s_ready + 16;                 // [2]
-  const uint32_t bar_o_done = bar_p_ready + 16;                  // [2]
+  const uint32_t bar_o_done = bar_p_ready + 16;                  // [2] O of a segment complete
+  const uint32_t bar_exp = bar_o_done + 16;                      // [2] exponentials of tile gt finished by group i
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   volatile int* abort_ptr = &abort_flag;
+  // softmax threads that own a real query row, rounded up to whole warps (they are tid 0 .. n_live-1)
+  const int n_live = (p.rows + 31) & ~31;
 
   // ---- set-up: lengths and tile prefix, barriers, TMEM
-  if (tid == 0) { abort_flag = 0; never_flag = 0; }
+  if (tid == 0) { abort_flag = 0; never_flag = 0; merge_is_last = 0; }
   for (int b = tid; b < p.batch; b += kThreads) {
     int Lc = p.cache_len[b];
     int Lq = p.q_len ? p.q_len[b] : p.q_cap;
@@ -201,18 +369,21 @@ attn_step_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
     }
     sched.prefix[p.batch] = acc;
     mbar_init(bar_q_full, 1);
-    mbar_init(bar_q_empty, 1);
+    mbar_init(bar_q_empty, (uint32_t)p.n_mt);       // one commit per MMA issuer
     mbar_init(bar_drain, 1);
+    mbar_init(bar_drain + 8, 1);
     for (int i = 0; i < KS; ++i) {
       mbar_init(bar_k_full + 8 * i, 1);
-      mbar_init(bar_k_empty + 8 * i, 1);
+      mbar_init(bar_k_empty + 8 * i, (uint32_t)p.n_mt);
       mbar_init(bar_v_full + 8 * i, 1);
-      mbar_init(bar_v_empty + 8 * i, 1);
+      mbar_init(bar_v_empty + 8 * i, (uint32_t)p.n_mt);
     }
     for (int i = 0; i < 2; ++i) {
+      const uint32_t live_i = (uint32_t)max(32, min(128, n_live - 128 * i));
       mbar_init(bar_s_ready + 8 * i, 1);
-      mbar_init(bar_p_ready + 8 * i, 128);
+      mbar_init(bar_p_ready + 8 * i, live_i);
       mbar_init(bar_o_done + 8 * i, 1);
+      mbar_init(bar_exp + 8 * i, live_i);
     }
     mbar_fence_init();
     fence_proxy_async_smem();
@@ -232,13 +403,26 @@ attn_step_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
   __syncthreads();
   tc_fence_after_sync();
   const uint32_t tmem = tmem_slot;
-  const int n_cta = gridDim.x;
+  // number of shares the item list is cut into (every share holds at least one item)
+  const int total_items = sched.prefix[p.batch] * p.nl * p.n_kv_heads;
+  const int n_cta = p.whole_units ? (int)gridDim.x : min((int)gridDim.x, total_items);
+  const bool has_work = p.whole_units || (int)blockIdx.x < n_cta;
+  if (!p.whole_units) {
+    for (int c = tid; c <= n_cta; c += kThreads)
+      sched.share_lo[c] = (int)((long long)total_items * c / max(n_cta, 1));
+    __syncthreads();
+  }
 
-  if (sched.prefix[p.batch] > 0 || p.whole_units) {
+  // The softmax warps keep a whole score row in registers; the other warpgroup needs few.
+  // setmaxnreg.inc waits, without a bound, until the registers it asks for are free: the host
+  // checks before the first launch that what the third warpgroup gives up covers what the two
+  // softmax warpgroups take (kRegsSoftmax, kRegsOther against the kernel's register count).
+  if (warp >= 8) {
+    setmaxnreg_dec<kRegsOther>();
     if (warp == 8) {
       // ================================================================= TMA producer
-      if (lane == 0) {
-        SegmentWalker walk(p, sched, blockIdx.x, n_cta);
+      if (lane == 0 && has_work) {
+        SegmentWalker walk(p, sched, blockIdx.x);
         Segment g;
         uint32_t kt = 0, vt = 0, seg = 0;
         bool ok = true;
@@ -290,23 +474,44 @@ attn_step_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
             mbar_wait(bar_v_full + 8 * (i % KS), (i / KS) & 1, &never_flag);
         }
       }
-    } else if (warp == 9) {
-      // ================================================================== MMA issuer
-      if (lane == 0) {
-        SegmentWalker walk(p, sched, blockIdx.x, n_cta);
+    } else if (warp == 9 || warp == 10) {
+      // ============================================ MMA issuers: warp 9 for M tile 0, warp 10 for M tile 1
+      // One thread per M tile, so that the scalar work around one tile's MMAs (barrier waits and
+      // commits) runs while the tensor pipe executes the other tile's.  The K, V and Q buffers are
+      // released when every issuer has committed (their "empty" barriers count n_mt arrivals).
+      const int mt = warp - 9;
+      if (lane == 0 && has_work && mt < p.n_mt) {
+        SegmentWalker walk(p, sched, blockIdx.x);
         Segment g;
         uint32_t kt = 0, vt = 0, gt = 0, seg = 0;
         bool ok = true;
         const uint32_t idesc_pv = make_idesc_bf16(128, D, 1);
-        // S[mt] = Q[mt] K^T for the tile in K stage `ks`, N = n16 keys
-        auto issue_s = [&](int mt, uint32_t ks, int n16) {
+        // descriptors of the first K-step of each operand buffer; the loops only add constants
+        const uint64_t desc_q = make_smem_desc_sw128(sm_q + mt * G::kTileBytes, 16, 1024);
+        const uint64_t desc_k0 = make_smem_desc_sw128(sm_k, 16, 1024);
+        const uint64_t desc_v0 = make_smem_desc_sw128(sm_v, kPanelBytes, 1024);
+        const uint32_t t_o = tmem + G::kColO + mt * D;
+        const uint32_t t_s = tmem + G::kColS + mt * 128;
+        // S = Q K^T for the tile in K stage `ks`, N = n16 keys
+        auto issue_s = [&](uint32_t ks, int n16) {
           const uint32_t idesc = make_idesc_bf16(128, (uint32_t)n16, 0);
-          const uint32_t d = tmem + G::kColS + mt * 128;
+          const uint64_t dk = desc_offset(desc_k0, ks * G::kTileBytes);
+          mma_ss<false>(t_s, desc_q, dk, idesc);
 #pragma unroll
-          for (int k = 0; k < D / 16; ++k) {
+          for (int k = 1; k < D / 16; ++k) {
             const uint32_t off = (k >> 2) * kPanelBytes + (k & 3) * 32;
-            mma_ss(d, make_smem_desc_sw128(sm_q + mt * G::kTileBytes + off, 16, 1024),
-                   make_smem_desc_sw128(sm_k + ks * G::kTileBytes + off, 16, 1024), idesc, k > 0 ? 1u : 0u);
+            mma_ss<true>(t_s, desc_offset(desc_q, off), desc_offset(dk, off), idesc);
+          }
+        };
+        // O (+)= P V for the tile in V stage `vs`, n16 keys
+        auto issue_pv = [&](uint32_t vs, int n16, bool first) {
+          const uint64_t dv = desc_offset(desc_v0, vs * G::kTileBytes);
+          if (first) mma_ts<false>(t_o, t_s, dv, idesc_pv); else mma_ts<true>(t_o, t_s, dv, idesc_pv);
+          if (n16 == kTileKeys) {
+#pragma unroll
+            for (int st = 1; st < kTileKeys / 16; ++st) mma_ts<true>(t_o, t_s + st * 8, desc_offset(dv, st * 2048), idesc_pv);
+          } else {
+            for (int st = 1; st < n16 / 16; ++st) mma_ts<true>(t_o, t_s + st * 8, desc_offset(dv, st * 2048), idesc_pv);
           }
         };
         while (ok && walk.next(g, n_cta)) {
@@ -319,11 +524,8 @@ attn_step_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
             ok = mbar_wait(bar_k_full + 8 * ks, (kt / KS) & 1, abort_ptr);
             if (!ok) break;
             tc_fence_after_sync();
-            const int n16 = (tile_valid(g, g.t_begin, p.fresh_box) + 15) & ~15;
-            for (int mt = 0; mt < p.n_mt; ++mt) {
-              issue_s(mt, ks, n16);
-              tc_commit(bar_s_ready + 8 * mt);
-            }
+            issue_s(ks, (tile_valid(g, g.t_begin, p.fresh_box) + 15) & ~15);
+            tc_commit(bar_s_ready + 8 * mt);
             tc_commit(bar_k_empty + 8 * ks);
             if (n == 1) tc_commit(bar_q_empty);
             ++kt;
@@ -333,36 +535,24 @@ attn_step_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
             const int n16 = (tile_valid(g, g.t_begin + it, p.fresh_box) + 15) & ~15;
             ok = mbar_wait(bar_v_full + 8 * vs, (vt / KS) & 1, abort_ptr);
             if (!ok) break;
-            const bool more = it + 1 < n;
-            uint32_t ks = 0;
-            int n16_next = 0;
-            for (int mt = 0; mt < p.n_mt && ok; ++mt) {
-              ok = mbar_wait(bar_p_ready + 8 * mt, gt & 1, abort_ptr);
+            ok = mbar_wait(bar_p_ready + 8 * mt, gt & 1, abort_ptr);
+            if (!ok) break;
+            tc_fence_after_sync();
+            issue_pv(vs, n16, it == 0);
+            if (it + 1 < n) {
+              tc_commit(bar_v_empty + 8 * vs);
+              const uint32_t ks = kt % KS;
+              ok = mbar_wait(bar_k_full + 8 * ks, (kt / KS) & 1, abort_ptr);
               if (!ok) break;
               tc_fence_after_sync();
-              const uint32_t d = tmem + G::kColO + mt * D;
-              const uint32_t a = tmem + G::kColS + mt * 128;
-              for (int st = 0; st < n16 / 16; ++st)
-                mma_ts(d, a + st * 8, make_smem_desc_sw128(sm_v + vs * G::kTileBytes + st * 2048, kPanelBytes, 1024),
-                       idesc_pv, (it > 0 || st > 0) ? 1u : 0u);
-              tc_commit(bar_o_done + 8 * mt);
-              if (mt == p.n_mt - 1) tc_commit(bar_v_empty + 8 * vs);
-              if (more) {
-                if (mt == 0) {
-                  ks = kt % KS;
-                  ok = mbar_wait(bar_k_full + 8 * ks, (kt / KS) & 1, abort_ptr);
-                  if (!ok) break;
-                  tc_fence_after_sync();
-                  n16_next = (tile_valid(g, g.t_begin + it + 1, p.fresh_box) + 15) & ~15;
-                }
-                issue_s(mt, ks, n16_next);
-                tc_commit(bar_s_ready + 8 * mt);
-                if (mt == p.n_mt - 1) {
-                  tc_commit(bar_k_empty + 8 * ks);
-                  if (it + 2 == n) tc_commit(bar_q_empty);
-                  ++kt;
-                }
-              }
+              issue_s(ks, (tile_valid(g, g.t_begin + it + 1, p.fresh_box) + 15) & ~15);
+              tc_commit(bar_s_ready + 8 * mt);   // also tells the softmax warps that P V of tile `it` is done
+              tc_commit(bar_k_empty + 8 * ks);
+              if (it + 2 == n) tc_commit(bar_q_empty);
+              ++kt;
+            } else {
+              tc_commit(bar_o_done + 8 * mt);      // O of the segment is complete
+              tc_commit(bar_v_empty + 8 * vs);
             }
             ++vt;
             ++gt;
@@ -370,57 +560,75 @@ attn_step_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
           ++seg;
         }
         // every MMA issued by this thread has finished before TMEM is released
-        tc_commit(bar_drain);
-        mbar_wait(bar_drain, 0, &never_flag);
+        tc_commit(bar_drain + 8 * mt);
+        mbar_wait(bar_drain + 8 * mt, 0, &never_flag);
       }
-    } else {
-      // ============================================================= softmax warpgroups
+    }
+  } else {
+    setmaxnreg_inc<kRegsSoftmax>();
+    if (tid < n_live) {
+      // ================================================= softmax warps (those that own real rows)
       const int mt = warp >> 2;
-      if (mt < p.n_mt) {
-        const int row = (warp & 3) * 32 + lane;                 // row of the M tile = TMEM lane
-        const uint32_t t_lane = (uint32_t)((warp & 3) * 32) << 16;
-        const uint32_t t_s = tmem + t_lane + G::kColS + mt * 128;
-        const uint32_t t_o = tmem + t_lane + G::kColO + mt * D;
-        const int r_unit = mt * 128 + row;                      // row within the unit
-        const bool real_row = r_unit < p.rows;
-        const int h_local = real_row ? r_unit / p.q_cap : 0;
-        const int i_row = real_row ? r_unit % p.q_cap : 0;
-        SegmentWalker walk(p, sched, blockIdx.x, n_cta);
+      const int row = (warp & 3) * 32 + lane;                 // row of the M tile = TMEM lane
+      const uint32_t t_lane = (uint32_t)((warp & 3) * 32) << 16;
+      const uint32_t t_s = tmem + t_lane + G::kColS + mt * 128;
+      const uint32_t t_o = tmem + t_lane + G::kColO + mt * D;
+      const int r_unit = mt * 128 + row;                      // row within the unit (== tid)
+      const bool real_row = r_unit < p.rows;
+      const int h_local = real_row ? r_unit / p.q_cap : 0;
+      const int i_row = real_row ? r_unit % p.q_cap : 0;
+      const int n_live_mt = min(128, n_live - 128 * mt);   // live softmax threads of this M tile
+      // the warp leaves a wait together, so the .sync.aligned TMEM instructions that follow
+      // always see a converged warp, also when a wait is given up
+      auto wait_warp = [&](uint32_t bar, uint32_t parity) {
+        return __all_sync(0xffffffffu, mbar_wait(bar, parity, abort_ptr)) != 0;
+      };
+      auto out_row_of = [&](int lc_layer, int b, int kvh, int hl, int ir) {
+        return (((size_t)lc_layer * p.batch + b) * p.n_q_heads + (size_t)kvh * p.group + hl) * p.q_cap + ir;
+      };
+      auto zero_my_row = [&](size_t qrow) {
+        if (real_row) {
+          uint4* o = reinterpret_cast<uint4*>(p.out + qrow * D);
+#pragma unroll
+          for (int c = 0; c < D / 8; ++c) o[c] = make_uint4(0, 0, 0, 0);
+          if (p.lse) p.lse[qrow] = -CUDART_INF_F;
+        }
+      };
+      if (!p.whole_units) {
+        // units without any key (inactive batch elements) appear in no share: zero them here
+        const int n_units = p.nl * p.n_kv_heads * p.batch;
+        for (int unit = blockIdx.x; unit < n_units; unit += gridDim.x) {
+          const int b = unit % p.batch, grp = unit / p.batch;
+          if (sched.prefix[b + 1] == sched.prefix[b])
+            zero_my_row(out_row_of(grp / p.n_kv_heads, b, grp % p.n_kv_heads, h_local, i_row));
+        }
+      }
+      if (has_work) {
+        SegmentWalker walk(p, sched, blockIdx.x);
         Segment g;
-        uint32_t gt = 0;
+        uint32_t gt = 0, seg = 0;
         bool ok = true;
-        uint32_t v[32];
-        // the warp leaves a wait together, so the .sync.aligned TMEM instructions that follow
-        // always see a converged warp, also when a wait is given up
-        auto wait_warp = [&](uint32_t bar, uint32_t parity) {
-          return __all_sync(0xffffffffu, mbar_wait(bar, parity, abort_ptr)) != 0;
-        };
         while (ok && walk.next(g, n_cta)) {
           const int n = g.t_end - g.t_begin;
-          const size_t qrow = (((size_t)g.lc_layer * p.batch + g.b) * p.n_q_heads + (size_t)g.kvh * p.group + h_local) *
-                                  p.q_cap + i_row;
+          const size_t qrow = out_row_of(g.lc_layer, g.b, g.kvh, h_local, i_row);
           if (n <= 0) {  // whole-unit mode, inactive batch element: the unit's rows are zero
-            if (real_row) {
-              uint4* o = reinterpret_cast<uint4*>(p.out + qrow * D);
-#pragma unroll
-              for (int c = 0; c < D / 8; ++c) o[c] = make_uint4(0, 0, 0, 0);
-              if (p.lse) p.lse[qrow] = -CUDART_INF_F;
-            }
+            zero_my_row(qrow);
             continue;
           }
-          float m_run = -CUDART_INF_F, l_run = 0.f;
+          float m_used = -CUDART_INF_F, l_run = 0.f;
           for (int it = 0; it < n && ok; ++it, ++gt) {
             const int valid = tile_valid(g, g.t_begin + it, p.fresh_box);
             const int n16 = (valid + 15) & ~15;
-            const int n_chunks = (valid + 31) >> 5;
-            if (mt == 0 && valid < n16) {
+            if (valid < n16) {
               // V rows in [valid, n16) would be multiplied by P = 0: clear them so that stale
-              // NaN / Inf bit patterns cannot reach O.
+              // NaN / Inf bit patterns cannot reach O.  Each M tile's warps do it before they
+              // announce their P, so it precedes that tile's P V product (the two tiles write the
+              // same zeros).
               const uint32_t vs = gt % KS;
               ok = wait_warp(bar_v_full + 8 * vs, (gt / KS) & 1);
               if (!ok) break;
               const int per_row = G::kPanels * 8;
-              for (int idx = tid; idx < (n16 - valid) * per_row; idx += 128) {
+              for (int idx = row; idx < (n16 - valid) * per_row; idx += n_live_mt) {
                 const int r = valid + idx / per_row, rem = idx % per_row;
                 const uint32_t a = sm_v + vs * G::kTileBytes + (rem >> 3) * kPanelBytes + r * 128 + (rem & 7) * 16;
                 asm volatile("st.shared.v4.b32 [%0], {%1, %1, %1, %1};" ::"r"(a), "r"(0u) : "memory");
@@ -430,68 +638,32 @@ attn_step_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
             ok = wait_warp(bar_s_ready + 8 * mt, gt & 1);
             if (!ok) break;
             tc_fence_after_sync();
-            // pass 1: row maximum over the valid keys of this tile
-            float mx = -CUDART_INF_F;
-            for (int c = 0; c < n_chunks; ++c) {
-              tmem_ld32(t_s + c * 32, v);
-              tmem_ld_wait();
-              if (c * 32 + 32 <= valid) {
-#pragma unroll
-                for (int j = 0; j < 32; ++j) mx = fmaxf(mx, __uint_as_float(v[j]));
-              } else {
-#pragma unroll
-                for (int j = 0; j < 32; ++j)
-                  if (c * 32 + j < valid) mx = fmaxf(mx, __uint_as_float(v[j]));
-              }
+            ExpTurn turn;
+            turn.abort_ptr = abort_ptr;
+            if (p.n_mt == 2) {
+              turn.wait_bar = (mt == 0) ? (gt > 0 ? bar_exp + 8 : 0u) : bar_exp;
+              turn.wait_parity = (mt == 0) ? (gt - 1) & 1 : gt & 1;
+              turn.arrive_bar = bar_exp + 8 * mt;
+            } else {
+              turn.wait_bar = turn.arrive_bar = 0;
+              turn.wait_parity = 0;
             }
-            const float m_new = fmaxf(m_run, mx * p.scale_log2);
-            if (it > 0 && __any_sync(0xffffffffu, m_new > m_run)) {
-              // some row of this warp has a new maximum: rescale the warp's O rows in TMEM
-              ok = wait_warp(bar_o_done + 8 * mt, (gt - 1) & 1);
-              if (!ok) break;
-              tc_fence_after_sync();
-              const float alpha = ex2_approx(m_run - m_new);
-#pragma unroll 1
-              for (int c = 0; c < D / 32; ++c) {
-                tmem_ld32(t_o + c * 32, v);
-                tmem_ld_wait();
-#pragma unroll
-                for (int j = 0; j < 32; ++j) v[j] = __float_as_uint(__uint_as_float(v[j]) * alpha);
-                tmem_st32(t_o + c * 32, v);
-              }
-              l_run *= alpha;
-            }
-            m_run = m_new;
-            // pass 2: P = 2^(s * scale - m), row sum, bf16 pairs written over S
-            float l_add = 0.f;
-            for (int c = 0; c < n_chunks; ++c) {
-              tmem_ld32(t_s + c * 32, v);
-              tmem_ld_wait();
-              uint32_t pk[16];
-#pragma unroll
-              for (int j = 0; j < 16; ++j) {
-                float p0 = ex2_approx(fmaf(__uint_as_float(v[2 * j]), p.scale_log2, -m_run));
-                float p1 = ex2_approx(fmaf(__uint_as_float(v[2 * j + 1]), p.scale_log2, -m_run));
-                if (c * 32 + 2 * j >= valid) p0 = 0.f;
-                if (c * 32 + 2 * j + 1 >= valid) p1 = 0.f;
-                const __nv_bfloat162 h = __floats2bfloat162_rn(p0, p1);
-                // the sum uses the rounded values the tensor core will multiply with
-                l_add += __low2float(h) + __high2float(h);
-                pk[j] = *reinterpret_cast<const uint32_t*>(&h);
-              }
-              tmem_st16(t_s + c * 16, pk);
-            }
-            l_run += l_add;
-            tmem_st_wait();
+            if (valid == kTileKeys)
+              ok = softmax_tile_full<D>(t_s, t_o, it == 0, p.scale_log2, m_used, l_run, turn);
+            else
+              ok = softmax_tile_ragged<D>(t_s, t_o, valid, it == 0, p.scale_log2, m_used, l_run, turn);
+            if (!ok) break;
             tc_fence_before_sync();
             mbar_arrive(bar_p_ready + 8 * mt);
           }
           if (!ok) break;
           // ---- epilogue of the segment: O is complete once the last P V product has finished
-          ok = wait_warp(bar_o_done + 8 * mt, (gt - 1) & 1);
+          ok = wait_warp(bar_o_done + 8 * mt, seg & 1);
+          ++seg;
           if (!ok) break;
           tc_fence_after_sync();
           const bool active = real_row && i_row < g.Lq;
+          uint32_t v[32];
           if (g.slot < 0) {
             const float inv = active ? 1.f / l_run : 0.f;
 #pragma unroll 1
@@ -515,22 +687,97 @@ attn_step_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
               }
             }
             if (real_row && p.lse)
-              p.lse[qrow] = active ? (m_run + lg2_approx(l_run)) * 0.6931471805599453f : -CUDART_INF_F;
+              p.lse[qrow] = active ? (m_used + lg2_approx(l_run)) * 0.6931471805599453f : -CUDART_INF_F;
           } else {
-            const size_t prow = ((size_t)g.slot * p.n_mt + mt) * 128 + row;
+            // ---- a piece of a split unit: leave (O, m, l) in the workspace; the block that completes
+            // the unit merges all pieces in block order, so the result does not depend on timing.
+            // Partial O is stored column-major per M tile ([D][128 rows]): a warp's 32 rows of one
+            // column are one 128-byte line, for the stores here and for the loads of the merge.
+            float* po = p.ws_o + ((size_t)g.slot * p.n_mt + mt) * (size_t)(D * 128) + row;
 #pragma unroll 1
             for (int c = 0; c < D / 32; ++c) {
               tmem_ld32(t_o + c * 32, v);
               tmem_ld_wait();
-              if (real_row) {
-                float4* o = reinterpret_cast<float4*>(p.ws_o + prow * D + c * 32);
 #pragma unroll
-                for (int q4 = 0; q4 < 8; ++q4)
-                  o[q4] = make_float4(__uint_as_float(v[4 * q4]), __uint_as_float(v[4 * q4 + 1]),
-                                      __uint_as_float(v[4 * q4 + 2]), __uint_as_float(v[4 * q4 + 3]));
+              for (int j = 0; j < 32; ++j) __stcg(po + (c * 32 + j) * 128, __uint_as_float(v[j]));
+            }
+            __stcg(reinterpret_cast<float2*>(p.ws_ml) + ((size_t)g.slot * p.n_mt + mt) * 128 + row,
+                   make_float2(m_used, l_run));
+            const UnitPieces up(p, sched, g, blockIdx.x);
+            const int n_pieces = up.c_last - up.c_first + 1;
+            const int unit = (g.lc_layer * p.n_kv_heads + g.kvh) * p.batch + g.b;
+            __threadfence();
+            named_bar_sync(1, n_live);
+            if (tid == 0) {
+              const unsigned int done = atomicAdd(p.tickets + unit, 1u);
+              merge_is_last = (done == (unsigned int)n_pieces - 1u) ? 1 : 0;
+              if (merge_is_last) p.tickets[unit] = 0;   // ready for the next launch
+            }
+            for (int i = tid; i < n_pieces; i += n_live) merge_slot[i] = up.slot_of(up.c_first + i);
+            named_bar_sync(1, n_live);
+            if (merge_is_last) {
+              __threadfence();
+              // every thread merges its own query row: first the maximum and the sum ...
+              float m_all = -CUDART_INF_F, l_all = 0.f;
+              for (int ib = 0; ib < n_pieces; ib += 4) {
+                float2 ml[4];
+#pragma unroll
+                for (int j = 0; j < 4; ++j)
+                  ml[j] = (ib + j < n_pieces)
+                              ? __ldcg(reinterpret_cast<const float2*>(p.ws_ml) +
+                                       ((size_t)merge_slot[ib + j] * p.n_mt + mt) * 128 + row)
+                              : make_float2(-CUDART_INF_F, 0.f);
+                const float m_new = fmaxf(fmaxf(fmaxf(ml[0].x, ml[1].x), fmaxf(ml[2].x, ml[3].x)), m_all);
+                l_all *= ex2_approx(m_all - m_new);
+#pragma unroll
+                for (int j = 0; j < 4; ++j) l_all += ml[j].y * ex2_approx(ml[j].x - m_new);
+                m_all = m_new;
+              }
+              const float inv = active ? 1.f / l_all : 0.f;
+              if (real_row && p.lse)
+                p.lse[qrow] = active ? (m_all + lg2_approx(l_all)) * 0.6931471805599453f : -CUDART_INF_F;
+              // ... then O, 32 columns at a time with the loads of two pieces in flight (the partial
+              // results sit in L2: latency, not bandwidth, would bound a narrower loop)
+#pragma unroll 1
+              for (int c = 0; c < D / 32; ++c) {
+                float acc[32];
+#pragma unroll
+                for (int j = 0; j < 32; ++j) acc[j] = 0.f;
+                for (int ib = 0; ib < n_pieces; ib += 2) {
+                  float x[2][32], w[2];
+#pragma unroll
+                  for (int i = 0; i < 2; ++i) {
+                    if (ib + i < n_pieces) {
+                      const size_t piece = (size_t)merge_slot[ib + i] * p.n_mt + mt;
+                      const float* src = p.ws_o + piece * (size_t)(D * 128) + row + (size_t)c * 32 * 128;
+#pragma unroll
+                      for (int j = 0; j < 32; ++j) x[i][j] = __ldcg(src + j * 128);
+                      w[i] = ex2_approx(__ldcg(p.ws_ml + (piece * 128 + row) * 2) - m_all);
+                    } else {
+#pragma unroll
+                      for (int j = 0; j < 32; ++j) x[i][j] = 0.f;
+                      w[i] = 0.f;
+                    }
+                  }
+#pragma unroll
+                  for (int j = 0; j < 32; ++j) acc[j] = fmaf(w[1], x[1][j], fmaf(w[0], x[0][j], acc[j]));
+                }
+                if (real_row) {
+                  uint4* o = reinterpret_cast<uint4*>(p.out + qrow * D + c * 32);
+#pragma unroll
+                  for (int q4 = 0; q4 < 4; ++q4) {
+                    uint32_t wd[4];
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) {
+                      const __nv_bfloat162 h = __floats2bfloat162_rn(active ? acc[q4 * 8 + 2 * j] * inv : 0.f,
+                                                                     active ? acc[q4 * 8 + 2 * j + 1] * inv : 0.f);
+                      wd[j] = *reinterpret_cast<const uint32_t*>(&h);
+                    }
+                    o[q4] = make_uint4(wd[0], wd[1], wd[2], wd[3]);
+                  }
+                }
               }
             }
-            if (real_row) *reinterpret_cast<float2*>(p.ws_ml + prow * 2) = make_float2(m_run, l_run);
           }
         }
       }
@@ -545,79 +792,6 @@ attn_step_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
     tc_fence_after_sync();
     tmem_dealloc(tmem, kTmemCols);
   }
-}
-
-// Merges the partial results of every unit that was split across blocks, in block order.
-template <int D>
-__global__ void __launch_bounds__(256)
-attn_combine_kernel(const AttnParams p, int n_cta) {
-  constexpr int E = D / 32;
-  const int unit = blockIdx.x;
-  const int r_unit = blockIdx.y * 8 + (threadIdx.x >> 5);
-  const int lane = threadIdx.x & 31;
-  if (r_unit >= p.rows) return;
-  const int grp = unit / p.batch, b = unit % p.batch;
-  const int lc_layer = grp / p.n_kv_heads, kvh = grp % p.n_kv_heads;
-  long long sum = 0, before = 0;
-  int T = 0, Lq_b = 0;
-  for (int bb = 0; bb < p.batch; ++bb) {
-    int Lc = max(0, min(p.cache_len[bb], p.capacity));
-    int Lq = max(0, min(p.q_len ? p.q_len[bb] : p.q_cap, p.q_cap));
-    const int t = tiles_of(Lc, Lq, p.fresh_box);
-    if (bb < b) before += t;
-    if (bb == b) { T = t; Lq_b = Lq; }
-    sum += t;
-  }
-  const int h_local = r_unit / p.q_cap, i_row = r_unit % p.q_cap;
-  const size_t qrow = (((size_t)lc_layer * p.batch + b) * p.n_q_heads + (size_t)kvh * p.group + h_local) * p.q_cap + i_row;
-  __nv_bfloat16* o = p.out + qrow * D + lane * E;
-  const long long total = sum * p.nl * p.n_kv_heads;
-  const long long u0 = (long long)grp * sum + before, u1 = u0 + T;
-  int c_first = 0, c_last = 0;
-  if (T > 0) {
-    c_first = (int)(u0 * n_cta / total);
-    while (total * (c_first + 1) / n_cta <= u0) ++c_first;
-    while (total * c_first / n_cta > u0) --c_first;
-    c_last = (int)((u1 - 1) * n_cta / total);
-    while (total * (c_last + 1) / n_cta <= u1 - 1) ++c_last;
-    while (total * c_last / n_cta > u1 - 1) --c_last;
-    if (c_first == c_last) return;   // the unit was computed whole by one block
-  }
-  if (T == 0 || i_row >= Lq_b) {
-#pragma unroll
-    for (int e = 0; e < E; ++e) o[e] = __float2bfloat16(0.f);
-    if (p.lse && lane == 0) p.lse[qrow] = -CUDART_INF_F;
-    return;
-  }
-  const int mt = r_unit >> 7, row = r_unit & 127;
-  float m_all = -CUDART_INF_F;
-  for (int c = c_first; c <= c_last; ++c) {
-    const long long r0 = total * c / n_cta;
-    const long long s0 = r0 > u0 ? r0 : u0;
-    if (s0 >= u1 || s0 >= total * (c + 1) / n_cta) continue;   // a block with an empty share
-    const int slot = (s0 == r0) ? 2 * c : 2 * c + 1;
-    m_all = fmaxf(m_all, p.ws_ml[(((size_t)slot * p.n_mt + mt) * 128 + row) * 2]);
-  }
-  float acc[E], l_all = 0.f;
-#pragma unroll
-  for (int e = 0; e < E; ++e) acc[e] = 0.f;
-  for (int c = c_first; c <= c_last; ++c) {
-    const long long r0 = total * c / n_cta;
-    const long long s0 = r0 > u0 ? r0 : u0;
-    if (s0 >= u1 || s0 >= total * (c + 1) / n_cta) continue;
-    const int slot = (s0 == r0) ? 2 * c : 2 * c + 1;
-    const size_t prow = ((size_t)slot * p.n_mt + mt) * 128 + row;
-    const float2 ml = *reinterpret_cast<const float2*>(p.ws_ml + prow * 2);
-    const float w = ex2_approx(ml.x - m_all);
-    l_all += w * ml.y;
-    const float* po = p.ws_o + prow * D + lane * E;
-#pragma unroll
-    for (int e = 0; e < E; ++e) acc[e] += w * po[e];
-  }
-  const float inv = 1.f / l_all;
-#pragma unroll
-  for (int e = 0; e < E; ++e) o[e] = __float2bfloat16(acc[e] * inv);
-  if (p.lse && lane == 0) p.lse[qrow] = (m_all + lg2_approx(l_all)) * 0.6931471805599453f;
 }
 
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
@@ -645,6 +819,15 @@ int encode_map(dlm_ctx* ctx, CUtensorMap* map, const void* base, int D, long lon
   return r == CUDA_SUCCESS ? DLM_OK : DLM_ERR_CUDA;
 }
 
+// The kernel starts with `numRegs` registers per thread in all 12 warps.  The 8 softmax warps then
+// ask for kRegsSoftmax each and block until they get them; only what the other 4 warps release
+// is certain to be free, so the request must fit inside that.
+bool register_budget_ok(const void* kern) {
+  cudaFuncAttributes a;
+  if (cudaFuncGetAttributes(&a, kern) != cudaSuccess) return false;
+  return a.numRegs >= kRegsOther && 8 * (kRegsSoftmax - a.numRegs) <= 4 * (a.numRegs - kRegsOther);
+}
+
 struct Plan {
   int n_mt, rows, grid, whole_units;
   size_t ws_o_bytes, ws_ml_bytes;
@@ -655,8 +838,9 @@ Plan make_plan(const dlm_ctx* ctx, const dlm_kv_cache* cache, int nl, int n_q_he
   pl.rows = (n_q_heads / cache->n_kv_heads) * q_cap;
   pl.n_mt = (pl.rows + 127) / 128;
   const long long units = (long long)nl * cache->batch * cache->n_kv_heads;
-  pl.whole_units = units >= 8LL * ctx->num_sms ? 1 : 0;
-  pl.grid = (int)(units < ctx->num_sms && pl.whole_units ? units : ctx->num_sms);
+  const int sms = ctx->num_sms < kMaxGrid ? ctx->num_sms : kMaxGrid;
+  pl.whole_units = (units >= 8LL * sms || units > kDlmMaxSplitUnits) ? 1 : 0;
+  pl.grid = (int)(units < sms && pl.whole_units ? units : sms);
   const size_t slots = pl.whole_units ? 0 : 2 * (size_t)pl.grid;
   pl.ws_o_bytes = slots * pl.n_mt * 128 * cache->head_dim * sizeof(float);
   pl.ws_ml_bytes = slots * pl.n_mt * 128 * 2 * sizeof(float);
@@ -698,6 +882,11 @@ extern "C" int dlm_freecache_attn_step(dlm_ctx* ctx, const dlm_kv_cache* cache, 
   const size_t need = dlm_attn_workspace_bytes(ctx, cache, nl, n_q_heads, q_cap);
   if (!workspace || workspace_bytes < need || ((uintptr_t)workspace & 255)) return DLM_ERR_WORKSPACE;
   const Plan pl = make_plan(ctx, cache, nl, n_q_heads, q_cap);
+  {  // the split schedule counts (unit, key tile) items in 32 bits
+    const long long tiles_per_unit = (cache->capacity + 127) / 128 + (q_cap + 127) / 128 + 1;
+    if (!pl.whole_units && (long long)nl * cache->batch * cache->n_kv_heads * tiles_per_unit >= (1LL << 30))
+      return DLM_ERR_UNSUPPORTED;
+  }
 
   AttnParams p;
   p.cache_len = cache->cache_len;
@@ -721,6 +910,7 @@ extern "C" int dlm_freecache_attn_step(dlm_ctx* ctx, const dlm_kv_cache* cache, 
   const float scale = softmax_scale > 0.f ? softmax_scale : 1.0f / sqrtf((float)D);
   p.scale_log2 = scale * 1.4426950408889634f;
   p.status = &ctx->words->status;
+  p.tickets = ctx->words->attn_unit_tickets;
 
   CUtensorMap tm_q, tm_kc, tm_vc, tm_kn, tm_vn;
   const long long slabs_new = (long long)nl * cache->batch * cache->n_kv_heads;
@@ -734,27 +924,24 @@ extern "C" int dlm_freecache_attn_step(dlm_ctx* ctx, const dlm_kv_cache* cache, 
   if (rc != DLM_OK) return rc;
 
   cudaStream_t s = static_cast<cudaStream_t>(stream);
-  const long long units = slabs_new;
   if (D == 128) {
     auto kern = attn_step_sm100_kernel<128>;
     static bool configured = false;
     if (!configured) {
+      if (!register_budget_ok(reinterpret_cast<const void*>(kern))) return DLM_ERR_UNSUPPORTED;
       DLM_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, Geometry<128>::kSmemBytes));
       configured = true;
     }
     kern<<<pl.grid, kThreads, Geometry<128>::kSmemBytes, s>>>(tm_q, tm_kc, tm_vc, tm_kn, tm_vn, p);
-    if (!pl.whole_units)
-      attn_combine_kernel<128><<<dim3((unsigned)units, (unsigned)((pl.rows + 7) / 8)), 256, 0, s>>>(p, pl.grid);
   } else {
     auto kern = attn_step_sm100_kernel<64>;
     static bool configured = false;
     if (!configured) {
+      if (!register_budget_ok(reinterpret_cast<const void*>(kern))) return DLM_ERR_UNSUPPORTED;
       DLM_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, Geometry<64>::kSmemBytes));
       configured = true;
     }
     kern<<<pl.grid, kThreads, Geometry<64>::kSmemBytes, s>>>(tm_q, tm_kc, tm_vc, tm_kn, tm_vn, p);
-    if (!pl.whole_units)
-      attn_combine_kernel<64><<<dim3((unsigned)units, (unsigned)((pl.rows + 7) / 8)), 256, 0, s>>>(p, pl.grid);
   }
-  return dlm_launch_ok(ctx, pl.whole_units ? 1 : 2);
+  return dlm_launch_ok(ctx, 1);
 }

@@ -9,12 +9,13 @@
 
 // Device words owned by a context.  `status` holds the first data-dependent error code
 // (0 = none); the ticket words let the last block of a kernel run a serial tail.
+constexpr int kDlmMaxSplitUnits = 2048;  // attention units that may be split across blocks in one call
 struct dlm_device_words {
   int status;
   unsigned int commit_ticket;
   unsigned int unmask_ticket;
-  unsigned int attn_ticket;
-  unsigned int pad[12];
+  unsigned int pad[13];
+  unsigned int attn_unit_tickets[kDlmMaxSplitUnits];  // pieces of a split unit finished so far
 };
 
 struct dlm_ctx {
