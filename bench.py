@@ -49,44 +49,63 @@ def measured_peaks():
 
 
 class ClockSampler:
-    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
-    Q = ("clocks.sm,clocks.max.sm,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
-         "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+    """Samples SM clocks and throttle reasons while the timed region runs (NVML reads only; falls back to
+    nvidia-smi when the NVML binding is missing)."""
+    REASONS = {0x8: "hw_slowdown", 0x40: "hw_thermal_slowdown", 0x20: "sw_thermal_slowdown", 0x4: "sw_power_cap"}
 
     def __init__(self, index):
-        self.index, self.proc, self.lines = index, None, []
+        self.index, self.sm, self.mx, self.reasons = index, [], None, set()
+        self._stop = threading.Event()
+        self.thread = None
+        self.note = None
+
+    def _loop(self):
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            h = pynvml.nvmlDeviceGetHandleByIndex(self.index)
+            self.mx = int(pynvml.nvmlDeviceGetMaxClockInfo(h, pynvml.NVML_CLOCK_SM))
+            while not self._stop.is_set():
+                self.sm.append(int(pynvml.nvmlDeviceGetClockInfo(h, pynvml.NVML_CLOCK_SM)))
+                r = int(pynvml.nvmlDeviceGetCurrentClocksEventReasons(h))
+                for bit, name in self.REASONS.items():
+                    if r & bit:
+                        self.reasons.add(name)
+                time.sleep(0.002)
+        except Exception as e:   # noqa: BLE001
+            self.note = f"nvml unavailable: {type(e).__name__}"
+            self._smi_once()
+
+    def _smi_once(self):
+        q = ("clocks.sm,clocks.max.sm,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+             "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        while not self._stop.is_set():
+            try:
+                out = subprocess.run(["nvidia-smi", "-i", str(self.index), f"--query-gpu={q}",
+                                      "--format=csv,noheader,nounits"], capture_output=True, text=True, timeout=5).stdout
+            except Exception:   # noqa: BLE001
+                return
+            f = [x.strip() for x in out.strip().split(",")]
+            if len(f) >= 6 and f[0].isdigit():
+                self.sm.append(int(f[0])); self.mx = int(f[1])
+                for n, v in zip(names, f[2:6]):
+                    if v.lower().startswith("active"):
+                        self.reasons.add(n)
 
     def start(self):
-        try:
-            self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.index), f"--query-gpu={self.Q}",
-                                          "--format=csv,noheader,nounits", "-lms", "100"],
-                                         stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
-            self.thread = threading.Thread(target=self._read, daemon=True)
-            self.thread.start()
-        except OSError:
-            self.proc = None
-
-    def _read(self):
-        for line in self.proc.stdout:
-            self.lines.append(line.strip())
+        self.thread = threading.Thread(target=self._loop, daemon=True)
+        self.thread.start()
 
     def stop(self):
-        if not self.proc:
-            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
-        self.proc.terminate()
-        self.thread.join(timeout=2)
-        sm, mx, reasons = [], [], set()
-        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
-        for line in self.lines:
-            f = [x.strip() for x in line.split(",")]
-            if len(f) < 6 or not f[0].isdigit():
-                continue
-            sm.append(int(f[0])); mx.append(int(f[1]))
-            for n, v in zip(names, f[2:6]):
-                if v.lower().startswith("active"):
-                    reasons.add(n)
-        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(mx) if mx else None,
-                "samples": len(sm), "reasons": sorted(reasons)}
+        self._stop.set()
+        if self.thread:
+            self.thread.join(timeout=10)
+        out = {"sm_mhz": statistics.median(self.sm) if self.sm else None, "sm_max_mhz": self.mx,
+               "samples": len(self.sm), "reasons": sorted(self.reasons)}
+        if self.note:
+            out["note"] = self.note
+        return out
 
 
 class Schedule:
@@ -155,34 +174,96 @@ class Workload:
         self.masked.zero_()
         self.masked[:, :st["n_masked"]] = 1
 
-    def launch_step(self, st, inputs=None, logits=None, attn_event=None):
-        """Enqueues one denoising step: attention (all layers), unmask, commit."""
+    def launch_attn(self, st, q, kn, vn):
         dlm, cfg = self.dlm, self.cfg
-        q, kn, vn = inputs if inputs is not None else self.pool[self.t % self.N_POOL]
-        lg = logits if logits is not None else self.logits[self.t % self.N_POOL]
         dlm.dlm_freecache_attn_step(self.ctx, self.cache, 0, cfg.n_layers, q, kn, vn, cfg.n_q_heads, cfg.block_len,
                                     None, 0.0, st["cache_len"], self.out, None, self.attn_ws)
-        if attn_event is not None:
-            attn_event.record()
+
+    def launch_rest(self, last, kn, vn, lg):
+        """Unmask, then the commit: the 4 staged rows, or the whole block when it completes."""
+        dlm, cfg = self.dlm, self.cfg
         dlm.dlm_unmask_select(self.ctx, lg, cfg.batch, cfg.block_len, cfg.vocab, self.masked, self.tokens, cfg.top_k,
                               self.tok, self.conf, self.sel_idx, self.n_sel, self.unmask_ws)
-        if st["last"]:      # block complete: freeze all of its rows and make them visible
+        if last:      # block complete: freeze all of its rows and make them visible
             dlm.dlm_kv_cache_commit(self.ctx, self.cache, kn, vn, cfg.block_len, None, None, dlm.DLM_DST_APPEND, None,
                                     cfg.block_len, 1, 0, cfg.n_layers)
-        else:               # stage the rows unmasked in this step at their own slots
+        else:         # stage the rows unmasked in this step at their own slots
             dlm.dlm_kv_cache_commit(self.ctx, self.cache, kn, vn, cfg.block_len, self.sel_idx, None,
                                     dlm.DLM_DST_WINDOW, self.n_sel, cfg.top_k, 0, 0, cfg.n_layers)
 
-    def run(self, steps, timed, e2e=False, host=None):
-        """Runs `steps` steps; returns (total_ms, attn_ms, attn_bytes, attn_flops)."""
-        tot = attn = 0.0
+    def launch_step(self, st, inputs=None, logits=None):
+        """Enqueues one denoising step through the C-ABI: attention (all layers), unmask, commit."""
+        q, kn, vn = inputs if inputs is not None else self.pool[self.t % self.N_POOL]
+        lg = logits if logits is not None else self.logits[self.t % self.N_POOL]
+        self.launch_attn(st, q, kn, vn)
+        self.launch_rest(st["last"], kn, vn, lg)
+
+    def capture(self):
+        """Captures the C-ABI calls of a step into CUDA graphs (the lengths and masks they read live in device
+        memory, so one capture serves every step): per input set one graph for the attention call and one for
+        unmask + commit in each of its two forms.  Replaying them removes the host's launch latency from the
+        device-side timing; the kernels and their arguments are exactly those of the direct calls."""
+        dlm = self.dlm
+        st = self.sched.at(0)
+        self.reset_block_state(st)
+        torch.cuda.synchronize()
+        self.g_attn, self.g_rest, self.n_attn, self.n_rest = [], [], [], []
+        side = torch.cuda.Stream()
+        for i in range(self.N_POOL):
+            q, kn, vn = self.pool[i]
+            g = torch.cuda.CUDAGraph()
+            c0 = dlm.dlm_launch_count(self.ctx)
+            with torch.cuda.graph(g, stream=side):
+                self.launch_attn(st, q, kn, vn)
+            self.g_attn.append(g)
+            self.n_attn.append(dlm.dlm_launch_count(self.ctx) - c0)
+            pair, counts = [], []
+            for last in (False, True):
+                g = torch.cuda.CUDAGraph()
+                c0 = dlm.dlm_launch_count(self.ctx)
+                with torch.cuda.graph(g, stream=side):
+                    self.launch_rest(last, kn, vn, self.logits[i])
+                pair.append(g)
+                counts.append(dlm.dlm_launch_count(self.ctx) - c0)
+            self.g_rest.append(pair)
+            self.n_rest.append(counts)
+        torch.cuda.synchronize()
+
+    def run_timed(self, steps):
+        """`steps` steps replayed from the graphs; L2 flushed before each; CUDA events on the launching stream
+        around the attention call and around the whole step (the flush is outside both).
+        Returns (total_ms, attn_ms, attn_bytes, attn_flops, kernel launches)."""
+        events, launches = [], 0
         nbytes = nflops = 0
         for _ in range(steps):
             st = self.sched.at(self.t)
-            if st["step_in_block"] == 0 or not timed:
+            if st["step_in_block"] == 0:
                 self.reset_block_state(st)
+            i = self.t % self.N_POOL
             self.flush.zero_()                      # evict L2 between timed steps
             e0, e1, e2 = (torch.cuda.Event(enable_timing=True) for _ in range(3))
+            e0.record()
+            self.g_attn[i].replay()
+            e1.record()
+            self.g_rest[i][1 if st["last"] else 0].replay()
+            e2.record()
+            events.append((e0, e1, e2))
+            launches += self.n_attn[i] + self.n_rest[i][1 if st["last"] else 0]
+            nbytes += attn_bytes(self.cfg, st["cache_len"])
+            nflops += attn_flops(self.cfg, st["cache_len"])
+            self.t += 1
+        torch.cuda.synchronize()
+        tot = sum(a.elapsed_time(c) for a, _, c in events)
+        attn = sum(a.elapsed_time(b) for a, b, _ in events)
+        return tot, attn, nbytes, nflops, launches
+
+    def run(self, steps, e2e=False, host=None):
+        """Direct (uncaptured) calls: warm-up, and the end-to-end leg with host buffers.  Returns wall ms."""
+        tot = 0.0
+        for _ in range(steps):
+            st = self.sched.at(self.t)
+            if st["step_in_block"] == 0 or not e2e:
+                self.reset_block_state(st)
             if e2e:
                 hq, hk, hv, hl, h_sel, h_n, h_tok = host
                 torch.cuda.synchronize()
@@ -196,16 +277,53 @@ class Workload:
                 torch.cuda.synchronize()
                 tot += (time.perf_counter() - t0) * 1e3
             else:
-                e0.record()
-                self.launch_step(st, attn_event=e1)
-                e2.record()
-                e2.synchronize()
-                tot += e0.elapsed_time(e2)
-                attn += e0.elapsed_time(e1)
-                nbytes += attn_bytes(self.cfg, st["cache_len"])
-                nflops += attn_flops(self.cfg, st["cache_len"])
+                self.launch_step(st)
             self.t += 1
-        return tot, attn, nbytes, nflops
+        torch.cuda.synchronize()
+        return tot
+
+    # ---- single-kernel measurements reported beside the step (same inputs, L2 flushed before each launch)
+    def time_call(self, fn, reps=10):
+        evs = []
+        for _ in range(reps):
+            self.flush.zero_()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record(); fn(); e1.record()
+            evs.append((e0, e1))
+        torch.cuda.synchronize()
+        ts = sorted(a.elapsed_time(b) for a, b in evs)
+        return ts[len(ts) // 2] * 1e-3
+
+    def other_kernels(self, peak_gbs):
+        """HBM-bound kernels of the path, each timed alone from a captured graph: the unmask pass over a fully
+        masked block and the cache refresh that (re)writes the whole prompt."""
+        dlm, cfg = self.dlm, self.cfg
+        B, Lblk, V = cfg.batch, cfg.block_len, cfg.vocab
+        side = torch.cuda.Stream()
+        res = {}
+        # unmask over all Lblk rows: k = 0 (propose only) keeps the mask full for every repetition
+        self.masked.fill_(1)
+        g = torch.cuda.CUDAGraph()
+        torch.cuda.synchronize()
+        with torch.cuda.graph(g, stream=side):
+            dlm.dlm_unmask_select(self.ctx, self.logits[0], B, Lblk, V, self.masked, self.tokens, 0, self.tok, self.conf,
+                                  None, None, self.unmask_ws)
+        t = self.time_call(g.replay)
+        nb = B * Lblk * V * 4
+        res["unmask_full_block"] = {"us": t * 1e6, "algorithmic_bytes": nb, "GB/s": nb / t / 1e9, "frac": nb / t / 1e9 / peak_gbs}
+        # prompt refresh: rows [0, prompt_len) of every layer rewritten from a source of the same shape
+        src_k = make_kv_rows((cfg.n_layers, B, cfg.n_kv_heads, cfg.prompt_len, cfg.head_dim), 5, self.dev)
+        src_v = make_kv_rows((cfg.n_layers, B, cfg.n_kv_heads, cfg.prompt_len, cfg.head_dim), 6, self.dev)
+        dst = torch.arange(cfg.prompt_len, dtype=torch.int32, device=self.dev).repeat(B, 1).contiguous()
+        g2 = torch.cuda.CUDAGraph()
+        torch.cuda.synchronize()
+        with torch.cuda.graph(g2, stream=side):
+            dlm.dlm_kv_cache_commit(self.ctx, self.cache, src_k, src_v, cfg.prompt_len, None, dst, dlm.DLM_DST_APPEND, None,
+                                    cfg.prompt_len, 0, 0, cfg.n_layers)
+        t = self.time_call(g2.replay)
+        nb = 2 * 2 * cfg.n_layers * B * cfg.n_kv_heads * cfg.prompt_len * cfg.head_dim * 2
+        res["commit_prompt_refresh"] = {"us": t * 1e6, "algorithmic_bytes": nb, "GB/s": nb / t / 1e9, "frac": nb / t / 1e9 / peak_gbs}
+        return res
 
 
 def cpu_oracle_sample(cfg, cfg_index, n_layers_sample):
@@ -242,7 +360,7 @@ def cpu_oracle_sample(cfg, cfg_index, n_layers_sample):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=64)
+    ap.add_argument("--steps", type=int, default=512)
     ap.add_argument("--warmup", type=int, default=8)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--config", default="dream7b")
@@ -256,7 +374,8 @@ def main():
                           f"{cfg.n_q_heads}q/{cfg.n_kv_heads}kv heads x {cfg.head_dim}, prompt {cfg.prompt_len} + {cfg.n_blocks} blocks of "
                           f"{cfg.block_len}, {cfg.steps_per_block} steps/block, vocab {cfg.vocab}, top-{cfg.top_k}",
               "attention_launch": "layer-batched (all layers in one call; synthetic stack)",
-              "l2": "flushed between timed steps (512 MB write)", "parallelism": f"replicated x{world} (independent sequences)"}
+              "l2": "flushed between timed steps (512 MB write, outside the timed events)",
+              "launch": "steps replayed from CUDA graphs captured from the C-ABI calls", "parallelism": f"replicated x{world} (independent sequences)"}
 
     if args.impl == "reference":
         if rank != 0:
@@ -295,14 +414,15 @@ def main():
             dist.barrier()
         torch.cuda.synchronize()
 
-    wl.run(max(args.warmup, 3), timed=False)
+    wl.run(max(args.warmup, 3))          # direct calls: first-use set-up happens here, outside any capture
+    wl.capture()
+    wl.t = 0
+    wl.run_timed(max(args.warmup, 3))
     wl.t = 0
     sampler = ClockSampler(local_rank)
     barrier()
     sampler.start()
-    launches0 = dlm.dlm_launch_count(wl.ctx)
-    tot_ms, attn_ms, nbytes, nflops = wl.run(args.steps, timed=True)
-    launches = dlm.dlm_launch_count(wl.ctx) - launches0
+    tot_ms, attn_ms, nbytes, nflops, launches = wl.run_timed(args.steps)
     barrier()
     clocks = sampler.stop()
     status = dlm.dlm_get_status(wl.ctx)
@@ -316,10 +436,10 @@ def main():
     h2d = sum(x.numel() * x.element_size() for x in host[:4])
     d2h = sum(x.numel() * x.element_size() for x in host[4:])
     wl.t = 0
-    wl.run(3, timed=False, e2e=True, host=host)
+    wl.run(3, e2e=True, host=host)
     wl.t = 0
-    e2e_steps = min(args.steps, 32)
-    e2e_ms, _, _, _ = wl.run(e2e_steps, timed=True, e2e=True, host=host)
+    e2e_steps = min(args.steps, 64)
+    e2e_ms = wl.run(e2e_steps, e2e=True, host=host)
 
     times = torch.tensor([tot_ms, attn_ms, e2e_ms], dtype=torch.float64, device=device)
     if world > 1:
@@ -344,6 +464,7 @@ def main():
                      "attn_us_per_launch": attn_ms * 1e3 / args.steps,
                      "attn_tflops": nflops / (attn_ms * 1e-3) / 1e12,
                      "algorithmic_bytes_per_launch": nbytes / args.steps},
+        "other_kernels": wl.other_kernels(peaks["hbm_gbs"]),
         "cpu_baseline": cpu_oracle_sample(cfg, cfg_index, 4),
     }
     print(json.dumps(line))
