@@ -9,12 +9,14 @@
 
 // Device words owned by a context.  `status` holds the first data-dependent error code
 // (0 = none); the ticket words let the last block of a kernel run a serial tail.
+constexpr int kDlmUnmaskTickets = 1024;  // batch elements whose selection can run in the tail of the reduce kernel
 constexpr int kDlmMaxSplitUnits = 2048;  // attention units that may be split across blocks in one call
 struct dlm_device_words {
   int status;
   unsigned int commit_ticket;
   unsigned int unmask_ticket;
   unsigned int pad[13];
+  unsigned int unmask_tickets[kDlmUnmaskTickets];     // blocks of a batch element finished so far
   unsigned int attn_unit_tickets[kDlmMaxSplitUnits];  // pieces of a split unit finished so far
 };
 

@@ -2,13 +2,15 @@
 // (Eq. 2: one logit row per masked position; Eq. 3: fill with the argmax;
 //  M_{t-1} = M_t \ U_t).
 //
-// Kernel 1 (vocab_reduce) is bound by HBM: only the logit rows of masked positions are read,
-// once, as 16-byte vectors.  A row is split into chunks of kChunk logits, one block per
-// (chunk, row); the block reduces its chunk to the triple (max, lowest argmax, sum of
-// exp(z - max)) with warp shuffles and writes it to the workspace.
-// Kernel 2 (unmask_select) runs one block per batch element: it merges the triples of each
-// row in chunk order (so the result does not depend on block scheduling and identical rows
-// give identical bits), then ranks the masked positions by (confidence desc, position asc).
+// vocab_reduce is bound by HBM: only the logit rows of masked positions are read, once, as
+// 16-byte vectors.  A row is split into chunks of kChunk logits, one block per (chunk, row); the
+// block reduces its chunk to the triple (max, lowest argmax, sum of exp(z - max)) with warp
+// shuffles and writes it to the workspace.  The last block of a batch element to finish (a
+// ticket counter) then runs the selection for that element in the same launch: one warp per row
+// merges the row's triples with a fixed shuffle tree (so the result does not depend on block
+// scheduling and identical rows give identical bits), then the masked positions are ranked by
+// (confidence desc, position asc).  Without ticket words (more batch elements than the context
+// has counters for, or the context-free entry point) the selection runs as a second kernel.
 #include <math_constants.h>
 
 #include "common.cuh"
@@ -17,7 +19,7 @@ namespace {
 
 constexpr int kThreads = 256;
 constexpr int kVecPerThread = 4;
-constexpr int kChunk = kThreads * kVecPerThread * 4;  // 4096 logits = 16 KB per block
+constexpr int kChunk = kThreads * kVecPerThread * 4;  // 4096 logits: the unit of the chunk length (and of workspace sizing)
 constexpr int kMaxBlockLen = 1024;
 
 struct Triple {
@@ -27,31 +29,43 @@ struct Triple {
   int pad;
 };
 
+struct SelectArgs {
+  int block_len, k;
+  uint8_t* masked;
+  int32_t* tokens;
+  int32_t* tok;
+  float* conf;
+  int32_t* sel_idx;
+  int32_t* n_sel;
+};
+
 __device__ __forceinline__ void take_better(float& m, int& i, float m2, int i2) {
   if (m2 > m || (m2 == m && i2 < i)) { m = m2; i = i2; }
 }
 
-__global__ void __launch_bounds__(kThreads)
-vocab_reduce_kernel(const float* __restrict__ logits, const uint8_t* __restrict__ masked, int vocab,
-                    int n_chunks, Triple* __restrict__ partial) {
-  const int row = blockIdx.y;
-  if (!masked[row]) return;
+// One block reduces chunk blockIdx.x (chunk_len logits) of logit row `row` to a Triple.  Every
+// thread streams its share with 8 independent 16-byte loads in flight and keeps a running
+// (max, lowest argmax, sum of exp(z - max)); the block combines them with a fixed tree.
+__device__ __forceinline__ void reduce_chunk(const float* __restrict__ logits, int vocab, int chunk_len, int n_chunks,
+                                             Triple* partial, int row) {
   const int chunk = blockIdx.x;
   const float* z = logits + (size_t)row * vocab;
-  const int begin = chunk * kChunk;
-  const int end = min(begin + kChunk, vocab);
+  const int begin = chunk * chunk_len;
+  const int end = min(begin + chunk_len, vocab);
   const int tid = threadIdx.x;
+  constexpr int U = 8;                       // vectors in flight per thread
+  constexpr int kStep = kThreads * 4 * U;    // logits per block iteration
 
-  float x[kVecPerThread * 4];
-  float m = -CUDART_INF_F;
+  float m = -CUDART_INF_F, s = 0.f;
   int mi = 0x7fffffff;
   const bool vec_ok = (((uintptr_t)(z + begin)) & 15) == 0;
-  if (vec_ok) {
-    // thread t owns vectors t, t + 256, ... of the chunk: ascending indices within a thread
+  for (int base = begin; base < end; base += kStep) {
+    float x[U * 4];
+    // thread t owns vectors t, t + 256, ... of the iteration: ascending indices within a thread
 #pragma unroll
-    for (int u = 0; u < kVecPerThread; ++u) {
-      const int e = begin + (u * kThreads + tid) * 4;
-      if (e + 3 < end) {
+    for (int u = 0; u < U; ++u) {
+      const int e = base + (u * kThreads + tid) * 4;
+      if (vec_ok && e + 3 < end) {
         const float4 v = __ldcs(reinterpret_cast<const float4*>(z + e));
         x[4 * u + 0] = v.x; x[4 * u + 1] = v.y; x[4 * u + 2] = v.z; x[4 * u + 3] = v.w;
       } else {
@@ -59,98 +73,140 @@ vocab_reduce_kernel(const float* __restrict__ logits, const uint8_t* __restrict_
         for (int c = 0; c < 4; ++c) x[4 * u + c] = (e + c < end) ? z[e + c] : -CUDART_INF_F;
       }
     }
+    float bm = m;
 #pragma unroll
-    for (int u = 0; u < kVecPerThread; ++u)
+    for (int u = 0; u < U; ++u)
 #pragma unroll
       for (int c = 0; c < 4; ++c)
-        if (x[4 * u + c] > m) { m = x[4 * u + c]; mi = begin + (u * kThreads + tid) * 4 + c; }
-  } else {
-    // rows whose chunk start is not 16-byte aligned (vocab not a multiple of 4): scalar loads
+        if (x[4 * u + c] > bm) { bm = x[4 * u + c]; mi = base + (u * kThreads + tid) * 4 + c; }
+    if (bm > m) {   // the running sum follows the running maximum
+      s *= __expf(m - bm);
+      m = bm;
+    }
+    if (m > -CUDART_INF_F) {
 #pragma unroll
-    for (int u = 0; u < kVecPerThread * 4; ++u) {
-      const int e = begin + u * kThreads + tid;
-      x[u] = (e < end) ? z[e] : -CUDART_INF_F;
-      if (x[u] > m) { m = x[u]; mi = e; }
+      for (int u = 0; u < U * 4; ++u) s += __expf(x[u] - m);
     }
   }
   // block maximum and its lowest index
+  float wm = m;
+  int wi = mi;
 #pragma unroll
   for (int o = 16; o > 0; o >>= 1) {
-    const float m2 = __shfl_xor_sync(0xffffffffu, m, o);
-    const int i2 = __shfl_xor_sync(0xffffffffu, mi, o);
-    take_better(m, mi, m2, i2);
+    const float m2 = __shfl_xor_sync(0xffffffffu, wm, o);
+    const int i2 = __shfl_xor_sync(0xffffffffu, wi, o);
+    take_better(wm, wi, m2, i2);
   }
   __shared__ float sm_m[kThreads / 32];
   __shared__ int sm_i[kThreads / 32];
   __shared__ float sm_s[kThreads / 32];
   const int warp = tid >> 5, lane = tid & 31;
-  if (lane == 0) { sm_m[warp] = m; sm_i[warp] = mi; }
+  if (lane == 0) { sm_m[warp] = wm; sm_i[warp] = wi; }
   __syncthreads();
   float bm = sm_m[0];
   int bi = sm_i[0];
 #pragma unroll
   for (int w = 1; w < kThreads / 32; ++w) take_better(bm, bi, sm_m[w], sm_i[w]);
-  // sum of exp(z - block max); an all -inf chunk contributes nothing
-  float s = 0.f;
-  if (bm > -CUDART_INF_F) {
+  // sums re-based on the block maximum; a thread that saw only -inf contributes nothing
+  float t = (m > -CUDART_INF_F) ? s * __expf(m - bm) : 0.f;
 #pragma unroll
-    for (int u = 0; u < kVecPerThread * 4; ++u) s += __expf(x[u] - bm);
-  }
-#pragma unroll
-  for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
-  if (lane == 0) sm_s[warp] = s;
+  for (int o = 16; o > 0; o >>= 1) t += __shfl_xor_sync(0xffffffffu, t, o);
+  if (lane == 0) sm_s[warp] = t;
   __syncthreads();
   if (tid == 0) {
     float total = 0.f;
 #pragma unroll
     for (int w = 0; w < kThreads / 32; ++w) total += sm_s[w];
-    Triple t;
-    t.m = bm; t.idx = bi; t.s = total; t.pad = 0;
-    partial[(size_t)row * n_chunks + chunk] = t;
+    __stcg(reinterpret_cast<int4*>(partial + (size_t)row * n_chunks + chunk),
+           make_int4(__float_as_int(bm), bi, __float_as_int(total), 0));
   }
 }
 
-__global__ void __launch_bounds__(kMaxBlockLen)
-unmask_select_kernel(const Triple* __restrict__ partial, int n_chunks, int block_len, int k,
-                     uint8_t* __restrict__ masked, int32_t* __restrict__ tokens,
-                     int32_t* __restrict__ tok, float* __restrict__ conf,
-                     int32_t* __restrict__ sel_idx, int32_t* __restrict__ n_sel) {
+// Selection for batch element b by the whole block (any block size that is a multiple of 32).
+// Reads the triples with L2 loads: other blocks of this launch wrote them.
+__device__ void select_batch(const Triple* partial, int n_chunks, int b, const SelectArgs& a) {
   __shared__ float s_conf[kMaxBlockLen];
+  __shared__ int32_t s_tok[kMaxBlockLen];
   __shared__ uint8_t s_sel[kMaxBlockLen];
   __shared__ int s_count;
-  const int b = blockIdx.x;
-  const int i = threadIdx.x;
-  const size_t p = (size_t)b * block_len + i;
-  bool is_masked = false;
-  int my_tok = -1;
-  float my_conf = -1.f;
-  if (i < block_len) {
-    is_masked = masked[p] != 0;
-    if (is_masked) {
-      const Triple* t = partial + p * n_chunks;
-      float m = -CUDART_INF_F;
-      int idx = 0;
-      for (int c = 0; c < n_chunks; ++c)
-        if (t[c].m > m) { m = t[c].m; idx = t[c].idx; }   // chunks ascend: strict > keeps the lowest index
-      float s = 0.f;
-      for (int c = 0; c < n_chunks; ++c)
-        if (t[c].m > -CUDART_INF_F) s += t[c].s * __expf(t[c].m - m);
-      my_tok = idx;
-      my_conf = 1.0f / s;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, n_warps = blockDim.x >> 5;
+  const int L = a.block_len, k = a.k;
+  const size_t p0 = (size_t)b * L;
+  if (tid == 0) s_count = 0;
+  // (1) one warp per row: merge the row's chunk triples (lanes stride over the chunks).  Rows are
+  // taken four at a time and each lane first loads its (up to) two triples of every one of them,
+  // so one L2 round trip serves four rows; rows with more than 64 chunks loop instead.
+  constexpr int RG = 4;
+  for (int i0 = warp * RG; i0 < L; i0 += n_warps * RG) {
+    int4 v[RG][2];
+    bool on[RG];
+#pragma unroll
+    for (int r = 0; r < RG; ++r) {
+      const int i = i0 + r;
+      on[r] = i < L && a.masked[p0 + i] != 0;   // uniform across the warp
+#pragma unroll
+      for (int h = 0; h < 2; ++h) {
+        const int c = lane + 32 * h;
+        v[r][h] = (on[r] && c < n_chunks)
+                      ? __ldcg(reinterpret_cast<const int4*>(partial + (p0 + i) * n_chunks) + c)
+                      : make_int4(__float_as_int(-CUDART_INF_F), 0x7fffffff, 0, 0);
+      }
     }
-    tok[p] = my_tok;
-    conf[p] = my_conf;
-    s_conf[i] = my_conf;
-    s_sel[i] = 0;
+#pragma unroll
+    for (int r = 0; r < RG; ++r) {
+      const int i = i0 + r;
+      if (i >= L) break;
+      int my_tok = -1;
+      float my_conf = -1.f;
+      if (on[r]) {
+        const int4* t = reinterpret_cast<const int4*>(partial + (p0 + i) * n_chunks);
+        float m = __int_as_float(v[r][0].x);
+        int idx = v[r][0].y;
+        take_better(m, idx, __int_as_float(v[r][1].x), v[r][1].y);
+        for (int c = lane + 64; c < n_chunks; c += 32) {
+          const int4 w = __ldcg(t + c);
+          take_better(m, idx, __int_as_float(w.x), w.y);
+        }
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) {
+          const float m2 = __shfl_xor_sync(0xffffffffu, m, o);
+          const int i2 = __shfl_xor_sync(0xffffffffu, idx, o);
+          take_better(m, idx, m2, i2);
+        }
+        float s = 0.f;
+#pragma unroll
+        for (int h = 0; h < 2; ++h) {
+          const float mc = __int_as_float(v[r][h].x);
+          if (mc > -CUDART_INF_F) s += __int_as_float(v[r][h].z) * __expf(mc - m);
+        }
+        for (int c = lane + 64; c < n_chunks; c += 32) {
+          const int4 w = __ldcg(t + c);
+          const float mc = __int_as_float(w.x);
+          if (mc > -CUDART_INF_F) s += __int_as_float(w.z) * __expf(mc - m);
+        }
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
+        my_tok = idx;
+        my_conf = 1.0f / s;
+      }
+      if (lane == 0) {
+        a.tok[p0 + i] = my_tok;
+        a.conf[p0 + i] = my_conf;
+        s_conf[i] = my_conf;
+        s_tok[i] = my_tok;
+        s_sel[i] = 0;
+      }
+    }
   }
   if (k <= 0) return;
-  if (i == 0) s_count = 0;
   __syncthreads();
-  // rank among the masked positions of this batch element: (confidence desc, position asc)
-  if (is_masked) {
+  // (2) rank among the masked positions of this batch element: (confidence desc, position asc)
+  for (int i = tid; i < L; i += blockDim.x) {
+    const float my_conf = s_conf[i];
+    if (my_conf < 0.f) continue;   // unmasked positions hold -1 < every confidence
     int rank = 0;
-    for (int j = 0; j < block_len; ++j) {
-      const float cj = s_conf[j];  // unmasked positions hold -1 < every confidence
+    for (int j = 0; j < L; ++j) {
+      const float cj = s_conf[j];
       rank += (cj > my_conf || (cj == my_conf && j < i)) ? 1 : 0;
     }
     if (rank < k) {
@@ -159,16 +215,63 @@ unmask_select_kernel(const Triple* __restrict__ partial, int n_chunks, int block
     }
   }
   __syncthreads();
-  if (i < block_len && s_sel[i]) {
+  for (int i = tid; i < L; i += blockDim.x) {
+    if (!s_sel[i]) continue;
     int order = 0;
     for (int j = 0; j < i; ++j) order += s_sel[j];
-    sel_idx[(size_t)b * k + order] = i;
-    tokens[p] = my_tok;
-    masked[p] = 0;
+    a.sel_idx[(size_t)b * k + order] = i;
+    a.tokens[p0 + i] = s_tok[i];
+    a.masked[p0 + i] = 0;
   }
   const int count = s_count;
-  for (int j = count + i; j < k; j += blockDim.x) sel_idx[(size_t)b * k + j] = -1;
-  if (i == 0) n_sel[b] = count;
+  for (int j = count + tid; j < k; j += blockDim.x) a.sel_idx[(size_t)b * k + j] = -1;
+  if (tid == 0) a.n_sel[b] = count;
+}
+
+__global__ void __launch_bounds__(kThreads)
+vocab_reduce_kernel(const float* __restrict__ logits, int vocab, int chunk_len, int n_chunks, Triple* partial,
+                    unsigned int* tickets, const SelectArgs sel) {
+  const int row = blockIdx.y;
+  if (sel.masked[row]) reduce_chunk(logits, vocab, chunk_len, n_chunks, partial, row);
+  if (tickets == nullptr) return;
+  // the last block of this batch element to get here runs its selection
+  __shared__ bool is_last;
+  const int b = row / sel.block_len;
+  __threadfence();
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    const unsigned int t = atomicAdd(tickets + b, 1u);
+    is_last = (t == (unsigned int)(n_chunks * sel.block_len) - 1u);
+    if (is_last) tickets[b] = 0;   // ready for the next launch
+  }
+  __syncthreads();
+  if (!is_last) return;
+  __threadfence();
+  select_batch(partial, n_chunks, b, sel);
+}
+
+__global__ void __launch_bounds__(kThreads)
+unmask_select_kernel(const Triple* partial, int n_chunks, const SelectArgs sel) {
+  select_batch(partial, n_chunks, blockIdx.x, sel);
+}
+
+int launch_unmask(const float* logits, int batch, int block_len, int vocab, uint8_t* masked, int32_t* tokens, int k,
+                  int32_t* tok, float* conf, int32_t* sel_idx, int32_t* n_sel, Triple* partial,
+                  unsigned int* tickets, cudaStream_t s) {
+  // Chunk length: a multiple of kChunk, grown until the grid is a few blocks per SM (the count of
+  // masked rows is only known on the device, so all rows count), at most 8 * kChunk.
+  int mult = (int)(((long long)vocab * batch * block_len / (4LL * 148)) / kChunk);
+  mult = mult < 1 ? 1 : (mult > 8 ? 8 : mult);
+  const int chunk_len = mult * kChunk;
+  const int n_chunks = (vocab + chunk_len - 1) / chunk_len;
+  SelectArgs a;
+  a.block_len = block_len; a.k = k; a.masked = masked; a.tokens = tokens; a.tok = tok; a.conf = conf;
+  a.sel_idx = sel_idx; a.n_sel = n_sel;
+  vocab_reduce_kernel<<<dim3(n_chunks, batch * block_len), kThreads, 0, s>>>(logits, vocab, chunk_len, n_chunks, partial,
+                                                                             tickets, a);
+  if (tickets != nullptr) return 1;
+  unmask_select_kernel<<<batch, kThreads, 0, s>>>(partial, n_chunks, a);
+  return 2;
 }
 
 }  // namespace
@@ -191,16 +294,11 @@ extern "C" int dlm_unmask_select(dlm_ctx* ctx, const float* logits, int batch, i
   if (((uintptr_t)logits & 3) != 0) return DLM_ERR_UNSUPPORTED;
   const size_t need = dlm_unmask_workspace_bytes(ctx, batch, block_len, vocab);
   if (!workspace || workspace_bytes < need || ((uintptr_t)workspace & 15)) return DLM_ERR_WORKSPACE;
-  const int n_chunks = (vocab + kChunk - 1) / kChunk;
-  cudaStream_t s = static_cast<cudaStream_t>(stream);
-  Triple* partial = static_cast<Triple*>(workspace);
-  vocab_reduce_kernel<<<dim3(n_chunks, batch * block_len), kThreads, 0, s>>>(logits, masked, vocab, n_chunks, partial);
-  const int threads = ((block_len + 31) / 32) * 32;
-  unmask_select_kernel<<<batch, threads, 0, s>>>(partial, n_chunks, block_len, k, masked, tokens, tok, conf,
-                                                 sel_idx, n_sel);
-  return dlm_launch_ok(ctx, 2);
+  unsigned int* tickets = batch <= kDlmUnmaskTickets ? ctx->words->unmask_tickets : nullptr;
+  const int n = launch_unmask(logits, batch, block_len, vocab, masked, tokens, k, tok, conf, sel_idx, n_sel,
+                              static_cast<Triple*>(workspace), tickets, static_cast<cudaStream_t>(stream));
+  return dlm_launch_ok(ctx, n);
 }
-
 // ---------------------------------------------------------------------------------------
 // dlm_unmask_select_static: the same two kernels with the per-row partial reductions kept in
 // a fixed device array that is part of the library image, for callers that cannot allocate
@@ -236,11 +334,7 @@ extern "C" int dlm_unmask_select_static(const float* logits, int batch, int bloc
       return DLM_ERR_CUDA;
     g_static_partial_addr[device] = addr;
   }
-  Triple* partial = g_static_partial_addr[device];
-  cudaStream_t s = static_cast<cudaStream_t>(stream);
-  vocab_reduce_kernel<<<dim3(n_chunks, batch * block_len), kThreads, 0, s>>>(logits, masked, vocab, n_chunks, partial);
-  const int threads = ((block_len + 31) / 32) * 32;
-  unmask_select_kernel<<<batch, threads, 0, s>>>(partial, n_chunks, block_len, k, masked, tokens, tok, conf,
-                                                 sel_idx, n_sel);
+  launch_unmask(logits, batch, block_len, vocab, masked, tokens, k, tok, conf, sel_idx, n_sel,
+                g_static_partial_addr[device], nullptr, static_cast<cudaStream_t>(stream));
   return cudaGetLastError() == cudaSuccess ? DLM_OK : DLM_ERR_CUDA;
 }
