@@ -13,7 +13,8 @@
 //   warp  8     TMA producer (one lane): Q once per segment, K and V tiles through two rings
 //   warp  9/10  tcgen05.mma issuer of M tile 0 / 1 (one lane each): S = Q K^T into TMEM, then
 //               O += P V with P read from TMEM (it overwrites S in place as packed bf16)
-//   warp  11    idle (fills the third warpgroup, which hands most of its registers over)
+//   warp  11    publisher (one lane): makes a finished partial result visible device-wide and
+//               bumps its unit's counter, so the softmax warps need not wait for that
 // Online softmax in fp32 with base-2 exponentials; a whole score row sits in registers between
 // the maximum and the exponentials; O stays in TMEM and is rescaled only when a row maximum has
 // grown by more than a threshold.
@@ -21,9 +22,12 @@
 // Scheduling.  Every (unit, key tile) pair is one item of a global list; block c takes the
 // contiguous share [c*T/G, (c+1)*T/G) of it.  A share covers whole units (result written
 // directly) and at most two partial units (unnormalised O, running max and sum written to the
-// workspace).  The block that finishes the last piece of a unit merges all its pieces, always
-// in block order, so the result is deterministic.  With many more units than SMs the split is
-// not worth its traffic and units are dealt round-robin instead.
+// workspace).  A block walks its share from the end to the start, so the piece at the start of a
+// share (the last piece of its unit) is the last thing the block computes; that block merges the
+// unit: it waits for the counter the other pieces' blocks bump after publishing their partial
+// results (they have lower block indices and computed those pieces first), then folds them into
+// its own O, which is still in TMEM, in block order: the result is deterministic.  With many
+// more units than SMs the split is not worth its traffic and units are dealt round-robin instead.
 #include <cuda.h>
 #include <cuda_bf16.h>
 #include <math_constants.h>
@@ -59,7 +63,7 @@ struct AttnParams {
   const int32_t* q_len;
   __nv_bfloat16* out;
   float* lse;
-  float* ws_o;    // [2 * grid][n_mt][D][128]    partial unnormalised O, column-major per M tile
+  float* ws_o;    // [2 * grid][n_mt][D/4][128][4]  partial unnormalised O: 4 columns of a row per 16-byte vector
   float* ws_ml;   // [2 * grid][n_mt][128][2]    partial (running max in log2 units, running sum)
   int nl, layer_begin, batch, n_kv_heads, n_q_heads, group, capacity, q_cap;
   int rows;        // group * q_cap: query rows per unit
@@ -84,6 +88,7 @@ struct Segment {
   int Lc, Lq, n_ct, T;    // lengths, cache tiles, total tiles of the unit
   int t_begin, t_end;     // tile range of this segment
   int slot;               // partial slot, or -1 when the segment is the whole unit
+  int merger;             // partial segment holding the unit's last tile: this block merges the unit
 };
 
 __device__ __forceinline__ int tiles_of(int Lc, int Lq, int fresh_box) {
@@ -96,15 +101,15 @@ __device__ __forceinline__ int tiles_of(int Lc, int Lq, int fresh_box) {
 struct SegmentWalker {
   const AttnParams& p;
   const Sched& s;
-  int pos, end, range_begin;
+  int end, range_begin;   // split mode: items [range_begin, end) are still to do
   int unit, n_units;
   __device__ SegmentWalker(const AttnParams& p_, const Sched& s_, int cta) : p(p_), s(s_) {
     n_units = p.nl * p.n_kv_heads * p.batch;
     if (p.whole_units) {
       unit = cta;
-      pos = end = range_begin = 0;
+      end = range_begin = 0;
     } else {
-      range_begin = pos = s.share_lo[cta];
+      range_begin = s.share_lo[cta];
       end = s.share_lo[cta + 1];
       unit = 0;
     }
@@ -123,13 +128,16 @@ struct SegmentWalker {
       g.t_begin = 0;
       g.t_end = g.T;
       g.slot = -1;
+      g.merger = 0;
       unit += n_cta;
       return true;
     }
-    if (pos >= end) return false;
+    // split mode: from the end of the share towards its start
+    if (end <= range_begin) return false;
     const int sum = s.prefix[p.batch];
-    const int grp = pos / sum;
-    const int rem = pos - grp * sum;
+    const int item = end - 1;
+    const int grp = item / sum;
+    const int rem = item - grp * sum;
     int b = 0;
     while (s.prefix[b + 1] <= rem) ++b;   // batch is small; units with zero tiles are skipped
     const int unit_start = grp * sum + s.prefix[b];
@@ -140,12 +148,13 @@ struct SegmentWalker {
     g.Lq = s.lq[b];
     g.T = s.prefix[b + 1] - s.prefix[b];
     g.n_ct = (g.Lc + kTileKeys - 1) / kTileKeys;
-    g.t_begin = pos - unit_start;
-    const int room = end - unit_start;
-    g.t_end = room < g.T ? room : g.T;
+    const int seg_lo = unit_start > range_begin ? unit_start : range_begin;
+    g.t_begin = seg_lo - unit_start;
+    g.t_end = end - unit_start;
     const bool whole = g.t_begin == 0 && g.t_end == g.T;
-    g.slot = whole ? -1 : (pos == range_begin ? 2 * (int)blockIdx.x : 2 * (int)blockIdx.x + 1);
-    pos = unit_start + g.t_end;
+    g.slot = whole ? -1 : (seg_lo == range_begin ? 2 * (int)blockIdx.x : 2 * (int)blockIdx.x + 1);
+    g.merger = (!whole && g.t_end == g.T) ? 1 : 0;
+    end = seg_lo;
     return true;
   }
 };
@@ -173,6 +182,24 @@ struct UnitPieces {
   // if the piece starts where the block's share starts, else its second one
   __device__ __forceinline__ int slot_of(int c) const { return s.share_lo[c] >= u0 ? 2 * c : 2 * c + 1; }
 };
+
+// Waits until the counter at `addr` reaches `target` (acquire, device scope).  Bounded like the
+// mbarrier waits: gives up after the same wall-time limit or when the block is aborting.
+__device__ __forceinline__ bool wait_counter(const unsigned int* addr, unsigned int target, volatile int* abort_flag) {
+  const uint64_t t0 = global_timer_ns();
+  for (uint32_t spin = 1;; ++spin) {
+    unsigned int v;
+    asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(addr) : "memory");
+    if (v >= target) return true;
+    if ((spin & 15u) == 0u) {
+      if (*abort_flag) return false;
+      if (global_timer_ns() - t0 > kWaitLimitNs) {
+        *abort_flag = 1;
+        return false;
+      }
+    }
+  }
+}
 
 // Softmax of one key tile for the query row held by this thread (S row in TMEM -> P row in TMEM).
 // O is rescaled only when the running maximum has grown by more than kRescaleThreshold (log2
@@ -326,7 +353,7 @@ attn_step_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
   __shared__ int abort_flag;
   __shared__ int never_flag;   // stays 0: for waits that must not be cut short by an abort
   __shared__ uint32_t tmem_slot;
-  __shared__ int merge_is_last;
+  __shared__ int merge_ok;
   __shared__ int merge_slot[kMaxGrid];
 
   const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
@@ -341,6 +368,7 @@ attn_step_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
   const uint32_t bar_p_ready = bar_s_ready + 16;                 // [2]
   const uint32_t bar_o_done = bar_p_ready + 16;                  // [2] O of a segment complete
   const uint32_t bar_exp = bar_o_done + 16;                      // [2] exponentials of tile gt finished by group i
+  const uint32_t bar_pub = bar_exp + 16;                         // partial result of a segment stored by every softmax thread
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   volatile int* abort_ptr = &abort_flag;
@@ -348,7 +376,7 @@ attn_step_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
   const int n_live = (p.rows + 31) & ~31;
 
   // ---- set-up: lengths and tile prefix, barriers, TMEM
-  if (tid == 0) { abort_flag = 0; never_flag = 0; merge_is_last = 0; }
+  if (tid == 0) { abort_flag = 0; never_flag = 0; merge_ok = 0; }
   for (int b = tid; b < p.batch; b += kThreads) {
     int Lc = p.cache_len[b];
     int Lq = p.q_len ? p.q_len[b] : p.q_cap;
@@ -372,6 +400,7 @@ attn_step_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
     mbar_init(bar_q_empty, (uint32_t)p.n_mt);       // one commit per MMA issuer
     mbar_init(bar_drain, 1);
     mbar_init(bar_drain + 8, 1);
+    mbar_init(bar_pub, (uint32_t)n_live);
     for (int i = 0; i < KS; ++i) {
       mbar_init(bar_k_full + 8 * i, 1);
       mbar_init(bar_k_empty + 8 * i, (uint32_t)p.n_mt);
@@ -563,6 +592,23 @@ attn_step_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
         tc_commit(bar_drain + 8 * mt);
         mbar_wait(bar_drain + 8 * mt, 0, &never_flag);
       }
+    } else {
+      // ================================================================= publisher (warp 11)
+      // A piece that some other block will merge: once every softmax thread has stored its row
+      // (they arrive on bar_pub and move on), make the stores visible device-wide and count the
+      // piece in its unit's counter.
+      if (lane == 0 && has_work && !p.whole_units) {
+        SegmentWalker walk(p, sched, blockIdx.x);
+        Segment g;
+        uint32_t pub = 0;
+        while (walk.next(g, n_cta)) {
+          if (g.slot < 0 || g.merger || g.t_end <= g.t_begin) continue;
+          if (!mbar_wait(bar_pub, pub & 1, abort_ptr)) break;
+          ++pub;
+          __threadfence();
+          atomicAdd(p.tickets + (g.lc_layer * p.n_kv_heads + g.kvh) * p.batch + g.b, 1u);
+        }
+      }
     }
   } else {
     setmaxnreg_inc<kRegsSoftmax>();
@@ -689,41 +735,45 @@ attn_step_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
             if (real_row && p.lse)
               p.lse[qrow] = active ? (m_used + lg2_approx(l_run)) * 0.6931471805599453f : -CUDART_INF_F;
           } else {
-            // ---- a piece of a split unit: leave (O, m, l) in the workspace; the block that completes
-            // the unit merges all pieces in block order, so the result does not depend on timing.
-            // Partial O is stored column-major per M tile ([D][128 rows]): a warp's 32 rows of one
-            // column are one 128-byte line, for the stores here and for the loads of the merge.
-            float* po = p.ws_o + ((size_t)g.slot * p.n_mt + mt) * (size_t)(D * 128) + row;
+            // ---- a piece of a split unit.  Partial O is stored as 16-byte vectors of 4 columns,
+            // [D/4][128 rows][4]: a warp's 32 rows of one vector are 512 contiguous bytes, for the
+            // stores here and for the loads of the merge.
+            if (!g.merger) {
+              float4* po = reinterpret_cast<float4*>(p.ws_o) + ((size_t)g.slot * p.n_mt + mt) * (size_t)(D / 4 * 128) + row;
 #pragma unroll 1
-            for (int c = 0; c < D / 32; ++c) {
-              tmem_ld32(t_o + c * 32, v);
-              tmem_ld_wait();
+              for (int c = 0; c < D / 32; ++c) {
+                tmem_ld32(t_o + c * 32, v);
+                tmem_ld_wait();
 #pragma unroll
-              for (int j = 0; j < 32; ++j) __stcg(po + (c * 32 + j) * 128, __uint_as_float(v[j]));
-            }
-            __stcg(reinterpret_cast<float2*>(p.ws_ml) + ((size_t)g.slot * p.n_mt + mt) * 128 + row,
-                   make_float2(m_used, l_run));
-            const UnitPieces up(p, sched, g, blockIdx.x);
-            const int n_pieces = up.c_last - up.c_first + 1;
-            const int unit = (g.lc_layer * p.n_kv_heads + g.kvh) * p.batch + g.b;
-            __threadfence();
-            named_bar_sync(1, n_live);
-            if (tid == 0) {
-              const unsigned int done = atomicAdd(p.tickets + unit, 1u);
-              merge_is_last = (done == (unsigned int)n_pieces - 1u) ? 1 : 0;
-              if (merge_is_last) p.tickets[unit] = 0;   // ready for the next launch
-            }
-            for (int i = tid; i < n_pieces; i += n_live) merge_slot[i] = up.slot_of(up.c_first + i);
-            named_bar_sync(1, n_live);
-            if (merge_is_last) {
+                for (int j = 0; j < 8; ++j)
+                  __stcg(po + (c * 8 + j) * 128, make_float4(__uint_as_float(v[4 * j]), __uint_as_float(v[4 * j + 1]),
+                                                             __uint_as_float(v[4 * j + 2]), __uint_as_float(v[4 * j + 3])));
+              }
+              __stcg(reinterpret_cast<float2*>(p.ws_ml) + ((size_t)g.slot * p.n_mt + mt) * 128 + row,
+                     make_float2(m_used, l_run));
+              mbar_arrive(bar_pub);   // the publisher warp takes it from here
+            } else {
+              // ---- the unit's last piece: this block merges.  The other pieces belong to blocks
+              // c_first .. this - 1, which computed them first thing; wait for their count, then fold
+              // them into O (own piece first, then block order: the result does not depend on timing).
+              const UnitPieces up(p, sched, g, blockIdx.x);
+              const int n_others = up.c_last - up.c_first;
+              const int unit = (g.lc_layer * p.n_kv_heads + g.kvh) * p.batch + g.b;
+              if (tid == 0) {
+                merge_ok = wait_counter(p.tickets + unit, (unsigned int)n_others, abort_ptr) ? 1 : 0;
+                if (merge_ok) p.tickets[unit] = 0;   // ready for the next launch
+              }
+              for (int i = tid; i < n_others; i += n_live) merge_slot[i] = up.slot_of(up.c_first + i);
+              named_bar_sync(1, n_live);
+              if (!merge_ok) { ok = false; break; }
               __threadfence();
-              // every thread merges its own query row: first the maximum and the sum ...
-              float m_all = -CUDART_INF_F, l_all = 0.f;
-              for (int ib = 0; ib < n_pieces; ib += 4) {
+              // maximum and sum over all pieces
+              float m_all = m_used, l_all = l_run;
+              for (int ib = 0; ib < n_others; ib += 4) {
                 float2 ml[4];
 #pragma unroll
                 for (int j = 0; j < 4; ++j)
-                  ml[j] = (ib + j < n_pieces)
+                  ml[j] = (ib + j < n_others)
                               ? __ldcg(reinterpret_cast<const float2*>(p.ws_ml) +
                                        ((size_t)merge_slot[ib + j] * p.n_mt + mt) * 128 + row)
                               : make_float2(-CUDART_INF_F, 0.f);
@@ -734,48 +784,50 @@ attn_step_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
                 m_all = m_new;
               }
               const float inv = active ? 1.f / l_all : 0.f;
+              const float w_own = ex2_approx(m_used - m_all);
               if (real_row && p.lse)
                 p.lse[qrow] = active ? (m_all + lg2_approx(l_all)) * 0.6931471805599453f : -CUDART_INF_F;
-              // ... then O, 32 columns at a time with the loads of two pieces in flight (the partial
-              // results sit in L2: latency, not bandwidth, would bound a narrower loop)
-#pragma unroll 1
-              for (int c = 0; c < D / 32; ++c) {
-                float acc[32];
+              // O: one other piece at a time, all of its row in flight at once (L2 latency, not
+              // bandwidth, bounds a narrower loop); the running sum lives in TMEM between pieces
+              for (int i = 0; i < n_others; ++i) {
+                const size_t piece = (size_t)merge_slot[i] * p.n_mt + mt;
+                const float4* src = reinterpret_cast<const float4*>(p.ws_o) + piece * (size_t)(D / 4 * 128) + row;
+                float4 x[D / 4];
 #pragma unroll
-                for (int j = 0; j < 32; ++j) acc[j] = 0.f;
-                for (int ib = 0; ib < n_pieces; ib += 2) {
-                  float x[2][32], w[2];
+                for (int j = 0; j < D / 4; ++j) x[j] = __ldcg(src + j * 128);
+                const float w = ex2_approx(__ldcg(p.ws_ml + (piece * 128 + row) * 2) - m_all);
+                const float w0 = (i == 0) ? w_own : 1.f;
+                const bool last = (i == n_others - 1);
 #pragma unroll
-                  for (int i = 0; i < 2; ++i) {
-                    if (ib + i < n_pieces) {
-                      const size_t piece = (size_t)merge_slot[ib + i] * p.n_mt + mt;
-                      const float* src = p.ws_o + piece * (size_t)(D * 128) + row + (size_t)c * 32 * 128;
+                for (int c = 0; c < D / 32; ++c) {
+                  tmem_ld32(t_o + c * 32, v);
+                  tmem_ld_wait();
 #pragma unroll
-                      for (int j = 0; j < 32; ++j) x[i][j] = __ldcg(src + j * 128);
-                      w[i] = ex2_approx(__ldcg(p.ws_ml + (piece * 128 + row) * 2) - m_all);
-                    } else {
+                  for (int j = 0; j < 8; ++j) {
+                    v[4 * j + 0] = __float_as_uint(fmaf(w, x[c * 8 + j].x, w0 * __uint_as_float(v[4 * j + 0])));
+                    v[4 * j + 1] = __float_as_uint(fmaf(w, x[c * 8 + j].y, w0 * __uint_as_float(v[4 * j + 1])));
+                    v[4 * j + 2] = __float_as_uint(fmaf(w, x[c * 8 + j].z, w0 * __uint_as_float(v[4 * j + 2])));
+                    v[4 * j + 3] = __float_as_uint(fmaf(w, x[c * 8 + j].w, w0 * __uint_as_float(v[4 * j + 3])));
+                  }
+                  if (!last) {
+                    tmem_st32(t_o + c * 32, v);
+                  } else if (real_row) {
+                    uint4* o = reinterpret_cast<uint4*>(p.out + qrow * D + c * 32);
 #pragma unroll
-                      for (int j = 0; j < 32; ++j) x[i][j] = 0.f;
-                      w[i] = 0.f;
+                    for (int q4 = 0; q4 < 4; ++q4) {
+                      uint32_t wd[4];
+#pragma unroll
+                      for (int j = 0; j < 4; ++j) {
+                        const __nv_bfloat162 h =
+                            __floats2bfloat162_rn(active ? __uint_as_float(v[q4 * 8 + 2 * j]) * inv : 0.f,
+                                                  active ? __uint_as_float(v[q4 * 8 + 2 * j + 1]) * inv : 0.f);
+                        wd[j] = *reinterpret_cast<const uint32_t*>(&h);
+                      }
+                      o[q4] = make_uint4(wd[0], wd[1], wd[2], wd[3]);
                     }
                   }
-#pragma unroll
-                  for (int j = 0; j < 32; ++j) acc[j] = fmaf(w[1], x[1][j], fmaf(w[0], x[0][j], acc[j]));
                 }
-                if (real_row) {
-                  uint4* o = reinterpret_cast<uint4*>(p.out + qrow * D + c * 32);
-#pragma unroll
-                  for (int q4 = 0; q4 < 4; ++q4) {
-                    uint32_t wd[4];
-#pragma unroll
-                    for (int j = 0; j < 4; ++j) {
-                      const __nv_bfloat162 h = __floats2bfloat162_rn(active ? acc[q4 * 8 + 2 * j] * inv : 0.f,
-                                                                     active ? acc[q4 * 8 + 2 * j + 1] * inv : 0.f);
-                      wd[j] = *reinterpret_cast<const uint32_t*>(&h);
-                    }
-                    o[q4] = make_uint4(wd[0], wd[1], wd[2], wd[3]);
-                  }
-                }
+                if (!last) tmem_st_wait();
               }
             }
           }
