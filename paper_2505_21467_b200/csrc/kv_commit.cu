@@ -66,16 +66,18 @@ __global__ void __launch_bounds__(kThreads) kv_commit_kernel(const CommitParams 
       rest /= p.n_kv_heads;
       const int b = (int)(rest % p.batch);
       const int lc = (int)(rest / p.batch);  // layer within the call
+      // the index words are read before the row count is checked (their slots always exist), so the
+      // three small loads are in flight together instead of one after the other
       const int len0 = p.cache_len[b];
+      const long long src = p.src_idx ? p.src_idx[(long long)b * p.n_max + r] : r;
+      const long long dst_given = p.dst_pos ? p.dst_pos[(long long)b * p.n_max + r] : 0;
       const int n = valid_rows(p, b, len0);
       if (n < 0) {
         if (r == 0 && vec == 0 && h == 0 && lc == 0) dlm_set_status(p.status, DLM_ERR_CAPACITY);
         continue;
       }
       if (r >= n) continue;
-      const long long src = p.src_idx ? p.src_idx[(long long)b * p.n_max + r] : r;
-      const long long dst = p.dst_pos ? p.dst_pos[(long long)b * p.n_max + r]
-                                      : (long long)len0 + (p.dst_mode == DLM_DST_WINDOW ? src : r);
+      const long long dst = p.dst_pos ? dst_given : (long long)len0 + (p.dst_mode == DLM_DST_WINDOW ? src : r);
       if (src < 0 || src >= p.src_len || dst < 0 || dst >= p.capacity) {
         if (vec == 0 && h == 0 && lc == 0) dlm_set_status(p.status, DLM_ERR_INDEX);
         continue;

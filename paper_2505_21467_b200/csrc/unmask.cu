@@ -44,8 +44,9 @@ __device__ __forceinline__ void take_better(float& m, int& i, float m2, int i2) 
 }
 
 // One block reduces chunk blockIdx.x (chunk_len logits) of logit row `row` to a Triple.  Every
-// thread streams its share with 8 independent 16-byte loads in flight and keeps a running
+// thread streams its share with U independent 16-byte loads in flight and keeps a running
 // (max, lowest argmax, sum of exp(z - max)); the block combines them with a fixed tree.
+template <int U>
 __device__ __forceinline__ void reduce_chunk(const float* __restrict__ logits, int vocab, int chunk_len, int n_chunks,
                                              Triple* partial, int row) {
   const int chunk = blockIdx.x;
@@ -53,7 +54,6 @@ __device__ __forceinline__ void reduce_chunk(const float* __restrict__ logits, i
   const int begin = chunk * chunk_len;
   const int end = min(begin + chunk_len, vocab);
   const int tid = threadIdx.x;
-  constexpr int U = 8;                       // vectors in flight per thread
   constexpr int kStep = kThreads * 4 * U;    // logits per block iteration
 
   float m = -CUDART_INF_F, s = 0.f;
@@ -228,25 +228,26 @@ __device__ void select_batch(const Triple* partial, int n_chunks, int b, const S
   if (tid == 0) a.n_sel[b] = count;
 }
 
+template <int U>
 __global__ void __launch_bounds__(kThreads)
 vocab_reduce_kernel(const float* __restrict__ logits, int vocab, int chunk_len, int n_chunks, Triple* partial,
                     unsigned int* tickets, const SelectArgs sel) {
   const int row = blockIdx.y;
-  if (sel.masked[row]) reduce_chunk(logits, vocab, chunk_len, n_chunks, partial, row);
+  if (sel.masked[row]) reduce_chunk<U>(logits, vocab, chunk_len, n_chunks, partial, row);
   if (tickets == nullptr) return;
   // the last block of this batch element to get here runs its selection
   __shared__ bool is_last;
+  // Thread 0 wrote this block's triple, so its release-acquire increment publishes it and, in
+  // the block that sees the full count, makes every other block's triple visible.
   const int b = row / sel.block_len;
-  __threadfence();
-  __syncthreads();
   if (threadIdx.x == 0) {
-    const unsigned int t = atomicAdd(tickets + b, 1u);
+    unsigned int t;
+    asm volatile("atom.acq_rel.gpu.global.add.u32 %0, [%1], 1;" : "=r"(t) : "l"(tickets + b) : "memory");
     is_last = (t == (unsigned int)(n_chunks * sel.block_len) - 1u);
     if (is_last) tickets[b] = 0;   // ready for the next launch
   }
   __syncthreads();
   if (!is_last) return;
-  __threadfence();
   select_batch(partial, n_chunks, b, sel);
 }
 
@@ -257,18 +258,24 @@ unmask_select_kernel(const Triple* partial, int n_chunks, const SelectArgs sel) 
 
 int launch_unmask(const float* logits, int batch, int block_len, int vocab, uint8_t* masked, int32_t* tokens, int k,
                   int32_t* tok, float* conf, int32_t* sel_idx, int32_t* n_sel, Triple* partial,
-                  unsigned int* tickets, cudaStream_t s) {
-  // Chunk length: a multiple of kChunk, grown until the grid is a few blocks per SM (the count of
-  // masked rows is only known on the device, so all rows count), at most 8 * kChunk.
-  int mult = (int)(((long long)vocab * batch * block_len / (4LL * 148)) / kChunk);
-  mult = mult < 1 ? 1 : (mult > 8 ? 8 : mult);
-  const int chunk_len = mult * kChunk;
+                  unsigned int* tickets, int num_sms, cudaStream_t s) {
+  // A pass of a block covers U * 1024 logits (U vectors in flight per thread); the smaller U
+  // when even one resident wave of blocks (4 per SM) would get less than 8192 logits each.
+  const long long wave = 4LL * (num_sms > 0 ? num_sms : 148);
+  const long long per_block = ((long long)vocab * batch * block_len + wave - 1) / wave;   // logits per block for one wave
+  const int U = per_block <= 4096 ? 4 : 8;   // both variants keep 4 blocks of 256 threads on an SM
+  // large problems: up to 4 passes per block (a couple of waves of fatter blocks stream better
+  // than many waves of one-pass blocks)
+  long long passes = per_block / (2 * 8192);
+  passes = passes < 1 ? 1 : (passes > 4 ? 4 : passes);
+  const int chunk_len = U * kThreads * 4 * (int)passes;
   const int n_chunks = (vocab + chunk_len - 1) / chunk_len;
   SelectArgs a;
   a.block_len = block_len; a.k = k; a.masked = masked; a.tokens = tokens; a.tok = tok; a.conf = conf;
   a.sel_idx = sel_idx; a.n_sel = n_sel;
-  vocab_reduce_kernel<<<dim3(n_chunks, batch * block_len), kThreads, 0, s>>>(logits, vocab, chunk_len, n_chunks, partial,
-                                                                             tickets, a);
+  const dim3 grid(n_chunks, batch * block_len);
+  if (U == 4) vocab_reduce_kernel<4><<<grid, kThreads, 0, s>>>(logits, vocab, chunk_len, n_chunks, partial, tickets, a);
+  else vocab_reduce_kernel<8><<<grid, kThreads, 0, s>>>(logits, vocab, chunk_len, n_chunks, partial, tickets, a);
   if (tickets != nullptr) return 1;
   unmask_select_kernel<<<batch, kThreads, 0, s>>>(partial, n_chunks, a);
   return 2;
@@ -296,7 +303,7 @@ extern "C" int dlm_unmask_select(dlm_ctx* ctx, const float* logits, int batch, i
   if (!workspace || workspace_bytes < need || ((uintptr_t)workspace & 15)) return DLM_ERR_WORKSPACE;
   unsigned int* tickets = batch <= kDlmUnmaskTickets ? ctx->words->unmask_tickets : nullptr;
   const int n = launch_unmask(logits, batch, block_len, vocab, masked, tokens, k, tok, conf, sel_idx, n_sel,
-                              static_cast<Triple*>(workspace), tickets, static_cast<cudaStream_t>(stream));
+                              static_cast<Triple*>(workspace), tickets, ctx->num_sms, static_cast<cudaStream_t>(stream));
   return dlm_launch_ok(ctx, n);
 }
 // ---------------------------------------------------------------------------------------
@@ -335,6 +342,6 @@ extern "C" int dlm_unmask_select_static(const float* logits, int batch, int bloc
     g_static_partial_addr[device] = addr;
   }
   launch_unmask(logits, batch, block_len, vocab, masked, tokens, k, tok, conf, sel_idx, n_sel,
-                g_static_partial_addr[device], nullptr, static_cast<cudaStream_t>(stream));
+                g_static_partial_addr[device], nullptr, 0, static_cast<cudaStream_t>(stream));
   return cudaGetLastError() == cudaSuccess ? DLM_OK : DLM_ERR_CUDA;
 }
