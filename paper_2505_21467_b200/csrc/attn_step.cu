@@ -53,7 +53,7 @@ struct Geometry {
   static constexpr int kPanels = D / 64;
   static constexpr int kTileBytes = kPanels * kPanelBytes;      // one K tile, V tile or Q M-tile
   static constexpr int kStages = (D == 128) ? 2 : 4;            // ring depth of K and of V
-  static constexpr int kSmemBytes = (2 + 2 * kStages) * kTileBytes + 1024 /*alignment*/ + 256 /*barriers*/;
+  static constexpr int kSmemBytes = (2 + 2 * kStages) * kTileBytes + 1024 /*alignment*/ + 512 /*barriers*/;
   static constexpr uint32_t kColO = 0;                          // O[mt] at mt * D
   static constexpr uint32_t kColS = 2 * D;                      // S[mt] at 2D + mt * 128 (P aliases it)
 };
@@ -201,37 +201,52 @@ __device__ __forceinline__ bool wait_counter(const unsigned int* addr, unsigned 
   }
 }
 
-// Softmax of one key tile for the query row held by this thread (S row in TMEM -> P row in TMEM).
+// A key tile is processed in half-steps of up to 64 keys.  Each M tile has two 64-column score
+// buffers in TMEM used alternately, so the scores of the half-step after next are computed by the
+// tensor pipe while the softmax warps work on the current one: they never wait for scores in the
+// steady state.  All roles enumerate the half-steps of a segment with this iterator.
+constexpr int kHalfKeys = 64;
+struct HalfStep {
+  int t;          // key tile
+  int k0;         // first key of the half-step within the tile (0 or 64)
+  int nkeys;      // valid keys (1..64)
+  bool first_of_tile, last_of_tile;
+};
+struct HalfIter {
+  const Segment& g;
+  int fresh_box, t, h;
+  __device__ HalfIter(const Segment& g_, int fresh_box_) : g(g_), fresh_box(fresh_box_), t(g_.t_begin), h(0) {}
+  __device__ __forceinline__ bool get(HalfStep& s) const {
+    if (t >= g.t_end) return false;
+    const int valid = tile_valid(g, t, fresh_box);
+    s.t = t;
+    s.k0 = h * kHalfKeys;
+    s.nkeys = min(kHalfKeys, valid - s.k0);
+    s.first_of_tile = (h == 0);
+    s.last_of_tile = (h == 1) || valid <= kHalfKeys;
+    return true;
+  }
+  __device__ __forceinline__ void advance(const HalfStep& s) {
+    if (s.last_of_tile) { ++t; h = 0; } else { h = 1; }
+  }
+};
+
+// Softmax of one half-step for the query row held by this thread (S row in TMEM -> P row in TMEM).
 // O is rescaled only when the running maximum has grown by more than kRescaleThreshold (log2
 // units): until then P is formed against the older, smaller maximum and may reach
 // 2^kRescaleThreshold, which bf16 and the fp32 accumulators hold just as well; the final division
 // by the row sum, taken against the same maximum, cancels it.
 constexpr float kRescaleThreshold = 8.0f;
 
-// With two M tiles the exponentials of the two softmax groups take turns on the SFU: group 1 starts
-// those of a tile when group 0 has finished its own, and group 0 starts the next tile's when
-// group 1 is done.  Left alone the two groups drift into lockstep, and then the SFU and the
-// tensor pipe idle in turn; alternating, one group's exponentials run under the other's MMAs.
-struct ExpTurn {
-  uint32_t wait_bar;      // 0: nothing to wait for
-  uint32_t wait_parity;
-  uint32_t arrive_bar;    // 0: nobody to tell
-  volatile int* abort_ptr;
-  __device__ __forceinline__ bool begin() const {
-    if (wait_bar == 0) return true;
-    return __all_sync(0xffffffffu, mbar_wait(wait_bar, wait_parity, abort_ptr)) != 0;
-  }
-  __device__ __forceinline__ void end() const {
-    if (arrive_bar != 0) mbar_arrive(arrive_bar);
-  }
-};
-
-// Rare path shared by both tile kinds: some row of the warp outgrew its maximum by more than the
-// threshold, so the warp's O rows in TMEM are rescaled (rows that did not grow keep factor 1).
-// The P V product of the previous tile has finished by then: its issuer commits the barrier that
-// announced this tile's scores only after that product.
+// Rare path shared by both kinds of half-step: some row of the warp outgrew its maximum by more
+// than the threshold, so the warp's O rows in TMEM are rescaled (rows that did not grow keep
+// factor 1).  The P V product of the previous half-step may still be running: wait for it first.
 template <int D>
-__device__ __noinline__ void rescale_o(uint32_t t_o, bool grow, float m_new, float& m_used, float& l_run) {
+__device__ __noinline__ bool rescale_o(uint32_t t_o, bool grow, float m_new, float& m_used, float& l_run,
+                                       uint32_t bar_pv_done, uint32_t parity, volatile int* abort_ptr) {
+  const bool ok = __all_sync(0xffffffffu, mbar_wait(bar_pv_done, parity, abort_ptr)) != 0;
+  if (!ok) return false;
+  tc_fence_after_sync();
   const float alpha = grow ? ex2_approx(m_used - m_new) : 1.0f;
   uint32_t v[32];
 #pragma unroll 1
@@ -242,24 +257,27 @@ __device__ __noinline__ void rescale_o(uint32_t t_o, bool grow, float m_new, flo
     for (int j = 0; j < 32; ++j) v[j] = __float_as_uint(__uint_as_float(v[j]) * alpha);
     tmem_st32(t_o + c * 32, v);
   }
+  tmem_st_wait();
   l_run *= alpha;
   if (grow) m_used = m_new;
+  return true;
 }
 
-// Full tile (128 valid keys): the whole score row sits in registers between the maximum and the
+// Full half-step (64 valid keys): the score row sits in registers between the maximum and the
 // exponentials, so TMEM is read once and with a single wait.
 template <int D>
-__device__ __forceinline__ bool softmax_tile_full(uint32_t t_s, uint32_t t_o, bool first, float scale_log2,
-                                                  float& m_used, float& l_run, const ExpTurn& turn) {
-  uint32_t s[128];
-#pragma unroll
-  for (int c = 0; c < 4; ++c) tmem_ld32(t_s + c * 32, s + 32 * c);
+__device__ __forceinline__ bool softmax_half_full(uint32_t t_s, uint32_t t_o, bool first, float scale_log2,
+                                                  float& m_used, float& l_run, uint32_t bar_pv_done,
+                                                  uint32_t pv_parity, volatile int* abort_ptr) {
+  uint32_t s[64];
+  tmem_ld32(t_s, s);
+  tmem_ld32(t_s + 32, s + 32);
   tmem_ld_wait();
   float mx[8];   // independent chains: the maximum is latency-bound otherwise
 #pragma unroll
   for (int c = 0; c < 8; ++c) mx[c] = __uint_as_float(s[c]);
 #pragma unroll
-  for (int j = 8; j < 128; j += 8) {
+  for (int j = 8; j < 64; j += 8) {
 #pragma unroll
     for (int c = 0; c < 8; ++c) mx[c] = fmaxf(mx[c], __uint_as_float(s[j + c]));
   }
@@ -270,12 +288,13 @@ __device__ __forceinline__ bool softmax_tile_full(uint32_t t_s, uint32_t t_o, bo
     l_run = 0.f;
   } else {
     const bool grow = m_new > m_used + kRescaleThreshold;
-    if (__any_sync(0xffffffffu, grow)) rescale_o<D>(t_o, grow, m_new, m_used, l_run);
+    if (__any_sync(0xffffffffu, grow)) {
+      if (!rescale_o<D>(t_o, grow, m_new, m_used, l_run, bar_pv_done, pv_parity, abort_ptr)) return false;
+    }
   }
-  if (!turn.begin()) return false;
   float l0 = 0.f, l1 = 0.f;
 #pragma unroll
-  for (int c = 0; c < 4; ++c) {
+  for (int c = 0; c < 2; ++c) {
     uint32_t pk[16];
 #pragma unroll
     for (int j = 0; j < 16; ++j) {
@@ -286,7 +305,6 @@ __device__ __forceinline__ bool softmax_tile_full(uint32_t t_s, uint32_t t_o, bo
       const __nv_bfloat162 h = __floats2bfloat162_rn(p0, p1);
       pk[j] = *reinterpret_cast<const uint32_t*>(&h);
     }
-    if (c == 3) turn.end();
     tmem_st16(t_s + c * 16, pk);
   }
   l_run += l0 + l1;
@@ -294,11 +312,12 @@ __device__ __forceinline__ bool softmax_tile_full(uint32_t t_s, uint32_t t_o, bo
   return true;
 }
 
-// Ragged tile (fewer than 128 valid keys: the end of the cache rows, or the fresh rows): 32 columns
-// at a time, keys at or beyond `valid` masked out.
+// Ragged half-step (fewer than 64 valid keys: the end of the cache rows, or the fresh rows): 32
+// columns at a time, keys at or beyond `valid` masked out.
 template <int D>
-__device__ __noinline__ bool softmax_tile_ragged(uint32_t t_s, uint32_t t_o, int valid, bool first, float scale_log2,
-                                                 float& m_used, float& l_run, const ExpTurn& turn) {
+__device__ __noinline__ bool softmax_half_ragged(uint32_t t_s, uint32_t t_o, int valid, bool first, float scale_log2,
+                                                 float& m_used, float& l_run, uint32_t bar_pv_done,
+                                                 uint32_t pv_parity, volatile int* abort_ptr) {
   const int n_chunks = (valid + 31) >> 5;
   uint32_t v[32];
   float mx = -CUDART_INF_F;
@@ -315,9 +334,10 @@ __device__ __noinline__ bool softmax_tile_ragged(uint32_t t_s, uint32_t t_o, int
     l_run = 0.f;
   } else {
     const bool grow = m_new > m_used + kRescaleThreshold;
-    if (__any_sync(0xffffffffu, grow)) rescale_o<D>(t_o, grow, m_new, m_used, l_run);
+    if (__any_sync(0xffffffffu, grow)) {
+      if (!rescale_o<D>(t_o, grow, m_new, m_used, l_run, bar_pv_done, pv_parity, abort_ptr)) return false;
+    }
   }
-  if (!turn.begin()) return false;
   float l_add = 0.f;
   for (int c = 0; c < n_chunks; ++c) {
     tmem_ld32(t_s + c * 32, v);
@@ -335,7 +355,6 @@ __device__ __noinline__ bool softmax_tile_ragged(uint32_t t_s, uint32_t t_o, int
     }
     tmem_st16(t_s + c * 16, pk);
   }
-  turn.end();
   l_run += l_add;
   tmem_st_wait();
   return true;
@@ -364,11 +383,12 @@ attn_step_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
   const uint32_t bar_q_full = sm_bar, bar_q_empty = sm_bar + 8, bar_drain = sm_bar + 16;   // drain: [2]
   const uint32_t bar_k_full = sm_bar + 32, bar_k_empty = bar_k_full + 8 * KS;
   const uint32_t bar_v_full = bar_k_empty + 8 * KS, bar_v_empty = bar_v_full + 8 * KS;
-  const uint32_t bar_s_ready = bar_v_empty + 8 * KS;             // [2]
-  const uint32_t bar_p_ready = bar_s_ready + 16;                 // [2]
-  const uint32_t bar_o_done = bar_p_ready + 16;                  // [2] O of a segment complete
-  const uint32_t bar_exp = bar_o_done + 16;                      // [2] exponentials of tile gt finished by group i
-  const uint32_t bar_pub = bar_exp + 16;                         // partial result of a segment stored by every softmax thread
+  const uint32_t bar_s_ready = bar_v_empty + 8 * KS;             // [M tile][score buffer]: scores of a half-step written
+  const uint32_t bar_p_ready = bar_s_ready + 32;                 // [M tile][score buffer]: P of a half-step written
+  const uint32_t bar_pv_done = bar_p_ready + 32;                 // [M tile][half-step parity] P V product finished.  Two P V
+                                                                 // products can be in flight, so consecutive half-steps use different
+                                                                 // barriers: a parity wait cannot tell phases two apart
+  const uint32_t bar_pub = bar_pv_done + 32;                     // partial result of a segment stored by every softmax thread
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   volatile int* abort_ptr = &abort_flag;
@@ -409,10 +429,12 @@ attn_step_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
     }
     for (int i = 0; i < 2; ++i) {
       const uint32_t live_i = (uint32_t)max(32, min(128, n_live - 128 * i));
-      mbar_init(bar_s_ready + 8 * i, 1);
-      mbar_init(bar_p_ready + 8 * i, live_i);
-      mbar_init(bar_o_done + 8 * i, 1);
-      mbar_init(bar_exp + 8 * i, live_i);
+      for (int u = 0; u < 2; ++u) {
+        mbar_init(bar_s_ready + 16 * i + 8 * u, 1);
+        mbar_init(bar_p_ready + 16 * i + 8 * u, live_i);
+      }
+      mbar_init(bar_pv_done + 16 * i, 1);
+      mbar_init(bar_pv_done + 16 * i + 8, 1);
     }
     mbar_fence_init();
     fence_proxy_async_smem();
@@ -521,70 +543,78 @@ attn_step_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
         const uint64_t desc_v0 = make_smem_desc_sw128(sm_v, kPanelBytes, 1024);
         const uint32_t t_o = tmem + G::kColO + mt * D;
         const uint32_t t_s = tmem + G::kColS + mt * 128;
-        // S = Q K^T for the tile in K stage `ks`, N = n16 keys
-        auto issue_s = [&](uint32_t ks, int n16) {
+        // S = Q K^T for the keys [k0, k0 + n16) of the tile in K stage `ks`, into score buffer `buf`
+        auto issue_s = [&](uint32_t ks, int k0, int n16, uint32_t buf) {
           const uint32_t idesc = make_idesc_bf16(128, (uint32_t)n16, 0);
-          const uint64_t dk = desc_offset(desc_k0, ks * G::kTileBytes);
-          mma_ss<false>(t_s, desc_q, dk, idesc);
+          const uint64_t dk = desc_offset(desc_k0, ks * G::kTileBytes + k0 * 128);
+          const uint32_t d = t_s + buf * kHalfKeys;
+          mma_ss<false>(d, desc_q, dk, idesc);
 #pragma unroll
           for (int k = 1; k < D / 16; ++k) {
             const uint32_t off = (k >> 2) * kPanelBytes + (k & 3) * 32;
-            mma_ss<true>(t_s, desc_offset(desc_q, off), desc_offset(dk, off), idesc);
+            mma_ss<true>(d, desc_offset(desc_q, off), desc_offset(dk, off), idesc);
           }
         };
-        // O (+)= P V for the tile in V stage `vs`, n16 keys
-        auto issue_pv = [&](uint32_t vs, int n16, bool first) {
-          const uint64_t dv = desc_offset(desc_v0, vs * G::kTileBytes);
-          if (first) mma_ts<false>(t_o, t_s, dv, idesc_pv); else mma_ts<true>(t_o, t_s, dv, idesc_pv);
-          if (n16 == kTileKeys) {
+        // O (+)= P V for the same keys, P in score buffer `buf`, V tile in stage `vs`
+        auto issue_pv = [&](uint32_t vs, int k0, int n16, uint32_t buf, bool first) {
+          const uint64_t dv = desc_offset(desc_v0, vs * G::kTileBytes + k0 * 128);
+          const uint32_t a = t_s + buf * kHalfKeys;
+          if (first) mma_ts<false>(t_o, a, dv, idesc_pv); else mma_ts<true>(t_o, a, dv, idesc_pv);
+          if (n16 == kHalfKeys) {
 #pragma unroll
-            for (int st = 1; st < kTileKeys / 16; ++st) mma_ts<true>(t_o, t_s + st * 8, desc_offset(dv, st * 2048), idesc_pv);
+            for (int st = 1; st < kHalfKeys / 16; ++st) mma_ts<true>(t_o, a + st * 8, desc_offset(dv, st * 2048), idesc_pv);
           } else {
-            for (int st = 1; st < n16 / 16; ++st) mma_ts<true>(t_o, t_s + st * 8, desc_offset(dv, st * 2048), idesc_pv);
+            for (int st = 1; st < n16 / 16; ++st) mma_ts<true>(t_o, a + st * 8, desc_offset(dv, st * 2048), idesc_pv);
           }
         };
+        uint32_t js = 0;   // half-steps whose scores have been issued (global count: buffer = js & 1)
         while (ok && walk.next(g, n_cta)) {
-          const int n = g.t_end - g.t_begin;
-          if (n <= 0) continue;
+          if (g.t_end <= g.t_begin) continue;
           ok = mbar_wait(bar_q_full, seg & 1, abort_ptr);
           if (!ok) break;
-          {  // prologue: S of the first tile
+          HalfIter si(g, p.fresh_box), pi(g, p.fresh_box);
+          // scores of the next half-step of the segment that has none yet, into buffer js & 1
+          auto issue_next_s = [&]() -> bool {
+            HalfStep hs;
+            if (!si.get(hs)) return true;
             const uint32_t ks = kt % KS;
-            ok = mbar_wait(bar_k_full + 8 * ks, (kt / KS) & 1, abort_ptr);
-            if (!ok) break;
-            tc_fence_after_sync();
-            issue_s(ks, (tile_valid(g, g.t_begin, p.fresh_box) + 15) & ~15);
-            tc_commit(bar_s_ready + 8 * mt);
-            tc_commit(bar_k_empty + 8 * ks);
-            if (n == 1) tc_commit(bar_q_empty);
-            ++kt;
-          }
-          for (int it = 0; it < n && ok; ++it) {
-            const uint32_t vs = vt % KS;
-            const int n16 = (tile_valid(g, g.t_begin + it, p.fresh_box) + 15) & ~15;
-            ok = mbar_wait(bar_v_full + 8 * vs, (vt / KS) & 1, abort_ptr);
-            if (!ok) break;
-            ok = mbar_wait(bar_p_ready + 8 * mt, gt & 1, abort_ptr);
-            if (!ok) break;
-            tc_fence_after_sync();
-            issue_pv(vs, n16, it == 0);
-            if (it + 1 < n) {
-              tc_commit(bar_v_empty + 8 * vs);
-              const uint32_t ks = kt % KS;
-              ok = mbar_wait(bar_k_full + 8 * ks, (kt / KS) & 1, abort_ptr);
-              if (!ok) break;
+            if (hs.first_of_tile) {
+              if (!mbar_wait(bar_k_full + 8 * ks, (kt / KS) & 1, abort_ptr)) return false;
               tc_fence_after_sync();
-              issue_s(ks, (tile_valid(g, g.t_begin + it + 1, p.fresh_box) + 15) & ~15);
-              tc_commit(bar_s_ready + 8 * mt);   // also tells the softmax warps that P V of tile `it` is done
-              tc_commit(bar_k_empty + 8 * ks);
-              if (it + 2 == n) tc_commit(bar_q_empty);
-              ++kt;
-            } else {
-              tc_commit(bar_o_done + 8 * mt);      // O of the segment is complete
-              tc_commit(bar_v_empty + 8 * vs);
             }
-            ++vt;
+            issue_s(ks, hs.k0, (hs.nkeys + 15) & ~15, js & 1);
+            tc_commit(bar_s_ready + 16 * mt + 8 * (js & 1));
+            ++js;
+            si.advance(hs);
+            if (hs.last_of_tile) {
+              tc_commit(bar_k_empty + 8 * ks);
+              ++kt;
+              if (si.t >= g.t_end) tc_commit(bar_q_empty);   // Q is not read again in this segment
+            }
+            return true;
+          };
+          ok = issue_next_s() && issue_next_s();   // both score buffers filled ahead
+          bool first = true;
+          HalfStep hs;
+          while (ok && pi.get(hs)) {
+            const uint32_t vs = vt % KS;
+            if (hs.first_of_tile) {
+              ok = mbar_wait(bar_v_full + 8 * vs, (vt / KS) & 1, abort_ptr);
+              if (!ok) break;
+            }
+            ok = mbar_wait(bar_p_ready + 16 * mt + 8 * (gt & 1), (gt >> 1) & 1, abort_ptr);
+            if (!ok) break;
+            tc_fence_after_sync();
+            issue_pv(vs, hs.k0, (hs.nkeys + 15) & ~15, gt & 1, first);
+            tc_commit(bar_pv_done + 16 * mt + 8 * (gt & 1));
+            first = false;
+            if (hs.last_of_tile) {
+              tc_commit(bar_v_empty + 8 * vs);
+              ++vt;
+            }
             ++gt;
+            pi.advance(hs);
+            ok = issue_next_s();   // the buffer just consumed takes the half-step after next
           }
           ++seg;
         }
@@ -652,7 +682,7 @@ attn_step_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
       if (has_work) {
         SegmentWalker walk(p, sched, blockIdx.x);
         Segment g;
-        uint32_t gt = 0, seg = 0;
+        uint32_t gt = 0, vt = 0;   // half-steps and key tiles done so far
         bool ok = true;
         while (ok && walk.next(g, n_cta)) {
           const int n = g.t_end - g.t_begin;
@@ -662,50 +692,51 @@ attn_step_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
             continue;
           }
           float m_used = -CUDART_INF_F, l_run = 0.f;
-          for (int it = 0; it < n && ok; ++it, ++gt) {
-            const int valid = tile_valid(g, g.t_begin + it, p.fresh_box);
-            const int n16 = (valid + 15) & ~15;
-            if (valid < n16) {
-              // V rows in [valid, n16) would be multiplied by P = 0: clear them so that stale
-              // NaN / Inf bit patterns cannot reach O.  Each M tile's warps do it before they
-              // announce their P, so it precedes that tile's P V product (the two tiles write the
-              // same zeros).
-              const uint32_t vs = gt % KS;
-              ok = wait_warp(bar_v_full + 8 * vs, (gt / KS) & 1);
-              if (!ok) break;
-              const int per_row = G::kPanels * 8;
-              for (int idx = row; idx < (n16 - valid) * per_row; idx += n_live_mt) {
-                const int r = valid + idx / per_row, rem = idx % per_row;
-                const uint32_t a = sm_v + vs * G::kTileBytes + (rem >> 3) * kPanelBytes + r * 128 + (rem & 7) * 16;
-                asm volatile("st.shared.v4.b32 [%0], {%1, %1, %1, %1};" ::"r"(a), "r"(0u) : "memory");
+          HalfIter hi(g, p.fresh_box);
+          HalfStep hs;
+          bool first = true;
+          while (ok && hi.get(hs)) {
+            if (hs.first_of_tile) {
+              const int valid = tile_valid(g, hs.t, p.fresh_box);
+              const int n16 = (valid + 15) & ~15;
+              if (valid < n16) {
+                // V rows in [valid, n16) would be multiplied by P = 0: clear them so that stale
+                // NaN / Inf bit patterns cannot reach O.  Each M tile's warps do it before they
+                // announce the P of the tile's first half-step, so it precedes that tile's P V
+                // products (the two M tiles write the same zeros).
+                const uint32_t vs = vt % KS;
+                ok = wait_warp(bar_v_full + 8 * vs, (vt / KS) & 1);
+                if (!ok) break;
+                const int per_row = G::kPanels * 8;
+                for (int idx = row; idx < (n16 - valid) * per_row; idx += n_live_mt) {
+                  const int r = valid + idx / per_row, rem = idx % per_row;
+                  const uint32_t a = sm_v + vs * G::kTileBytes + (rem >> 3) * kPanelBytes + r * 128 + (rem & 7) * 16;
+                  asm volatile("st.shared.v4.b32 [%0], {%1, %1, %1, %1};" ::"r"(a), "r"(0u) : "memory");
+                }
+                fence_proxy_async_smem();
               }
-              fence_proxy_async_smem();
             }
-            ok = wait_warp(bar_s_ready + 8 * mt, gt & 1);
+            const uint32_t buf = gt & 1;
+            ok = wait_warp(bar_s_ready + 16 * mt + 8 * buf, (gt >> 1) & 1);
             if (!ok) break;
             tc_fence_after_sync();
-            ExpTurn turn;
-            turn.abort_ptr = abort_ptr;
-            if (p.n_mt == 2) {
-              turn.wait_bar = (mt == 0) ? (gt > 0 ? bar_exp + 8 : 0u) : bar_exp;
-              turn.wait_parity = (mt == 0) ? (gt - 1) & 1 : gt & 1;
-              turn.arrive_bar = bar_exp + 8 * mt;
-            } else {
-              turn.wait_bar = turn.arrive_bar = 0;
-              turn.wait_parity = 0;
-            }
-            if (valid == kTileKeys)
-              ok = softmax_tile_full<D>(t_s, t_o, it == 0, p.scale_log2, m_used, l_run, turn);
+            if (hs.nkeys == kHalfKeys)
+              ok = softmax_half_full<D>(t_s + buf * kHalfKeys, t_o, first, p.scale_log2, m_used, l_run,
+                                        bar_pv_done + 16 * mt + 8 * ((gt - 1) & 1), ((gt - 1) >> 1) & 1, abort_ptr);
             else
-              ok = softmax_tile_ragged<D>(t_s, t_o, valid, it == 0, p.scale_log2, m_used, l_run, turn);
+              ok = softmax_half_ragged<D>(t_s + buf * kHalfKeys, t_o, hs.nkeys, first, p.scale_log2, m_used, l_run,
+                                          bar_pv_done + 16 * mt + 8 * ((gt - 1) & 1), ((gt - 1) >> 1) & 1, abort_ptr);
             if (!ok) break;
             tc_fence_before_sync();
-            mbar_arrive(bar_p_ready + 8 * mt);
+            mbar_arrive(bar_p_ready + 16 * mt + 8 * buf);
+            first = false;
+            ++gt;
+            if (hs.last_of_tile) ++vt;
+            hi.advance(hs);
           }
           if (!ok) break;
           // ---- epilogue of the segment: O is complete once the last P V product has finished
-          ok = wait_warp(bar_o_done + 8 * mt, seg & 1);
-          ++seg;
+          ok = wait_warp(bar_pv_done + 16 * mt + 8 * ((gt - 1) & 1), ((gt - 1) >> 1) & 1);
           if (!ok) break;
           tc_fence_after_sync();
           const bool active = real_row && i_row < g.Lq;
