@@ -527,11 +527,17 @@ attn_step_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
       }
     } else if (warp == 9 || warp == 10) {
       // ============================================ MMA issuers: warp 9 for M tile 0, warp 10 for M tile 1
-      // One thread per M tile, so that the scalar work around one tile's MMAs (barrier waits and
-      // commits) runs while the tensor pipe executes the other tile's.  The K, V and Q buffers are
+      // One warp per M tile, so that the scalar work around one tile's MMAs (barrier waits and
+      // commits) runs while the tensor pipe executes the other tile's.  The whole warp runs the
+      // loop and one elected lane issues: in warp-uniform code the descriptors live in uniform
+      // registers, which is what tcgen05.mma reads; issued from a divergent single-lane branch
+      // every MMA paid for moving its operands there.  The K, V and Q buffers are
       // released when every issuer has committed (their "empty" barriers count n_mt arrivals).
       const int mt = warp - 9;
-      if (lane == 0 && has_work && mt < p.n_mt) {
+      if (has_work && mt < p.n_mt) {
+        auto wait_warp = [&](uint32_t bar, uint32_t parity) {
+          return __all_sync(0xffffffffu, mbar_wait(bar, parity, abort_ptr)) != 0;
+        };
         SegmentWalker walk(p, sched, blockIdx.x);
         Segment g;
         uint32_t kt = 0, vt = 0, gt = 0, seg = 0;
@@ -548,29 +554,39 @@ attn_step_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
           const uint32_t idesc = make_idesc_bf16(128, (uint32_t)n16, 0);
           const uint64_t dk = desc_offset(desc_k0, ks * G::kTileBytes + k0 * 128);
           const uint32_t d = t_s + buf * kHalfKeys;
-          mma_ss<false>(d, desc_q, dk, idesc);
+          if (elect_one_sync()) {
+            mma_ss<false>(d, desc_q, dk, idesc);
 #pragma unroll
-          for (int k = 1; k < D / 16; ++k) {
-            const uint32_t off = (k >> 2) * kPanelBytes + (k & 3) * 32;
-            mma_ss<true>(d, desc_offset(desc_q, off), desc_offset(dk, off), idesc);
+            for (int k = 1; k < D / 16; ++k) {
+              const uint32_t off = (k >> 2) * kPanelBytes + (k & 3) * 32;
+              mma_ss<true>(d, desc_offset(desc_q, off), desc_offset(dk, off), idesc);
+            }
           }
+          __syncwarp();
         };
         // O (+)= P V for the same keys, P in score buffer `buf`, V tile in stage `vs`
         auto issue_pv = [&](uint32_t vs, int k0, int n16, uint32_t buf, bool first) {
           const uint64_t dv = desc_offset(desc_v0, vs * G::kTileBytes + k0 * 128);
           const uint32_t a = t_s + buf * kHalfKeys;
-          if (first) mma_ts<false>(t_o, a, dv, idesc_pv); else mma_ts<true>(t_o, a, dv, idesc_pv);
-          if (n16 == kHalfKeys) {
+          if (elect_one_sync()) {
+            if (first) mma_ts<false>(t_o, a, dv, idesc_pv); else mma_ts<true>(t_o, a, dv, idesc_pv);
+            if (n16 == kHalfKeys) {
 #pragma unroll
-            for (int st = 1; st < kHalfKeys / 16; ++st) mma_ts<true>(t_o, a + st * 8, desc_offset(dv, st * 2048), idesc_pv);
-          } else {
-            for (int st = 1; st < n16 / 16; ++st) mma_ts<true>(t_o, a + st * 8, desc_offset(dv, st * 2048), idesc_pv);
+              for (int st = 1; st < kHalfKeys / 16; ++st) mma_ts<true>(t_o, a + st * 8, desc_offset(dv, st * 2048), idesc_pv);
+            } else {
+              for (int st = 1; st < n16 / 16; ++st) mma_ts<true>(t_o, a + st * 8, desc_offset(dv, st * 2048), idesc_pv);
+            }
           }
+          __syncwarp();
+        };
+        auto commit = [&](uint32_t bar) {
+          if (elect_one_sync()) tc_commit(bar);
+          __syncwarp();
         };
         uint32_t js = 0;   // half-steps whose scores have been issued (global count: buffer = js & 1)
         while (ok && walk.next(g, n_cta)) {
           if (g.t_end <= g.t_begin) continue;
-          ok = mbar_wait(bar_q_full, seg & 1, abort_ptr);
+          ok = wait_warp(bar_q_full, seg & 1);
           if (!ok) break;
           HalfIter si(g, p.fresh_box), pi(g, p.fresh_box);
           // scores of the next half-step of the segment that has none yet, into buffer js & 1
@@ -579,17 +595,17 @@ attn_step_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
             if (!si.get(hs)) return true;
             const uint32_t ks = kt % KS;
             if (hs.first_of_tile) {
-              if (!mbar_wait(bar_k_full + 8 * ks, (kt / KS) & 1, abort_ptr)) return false;
+              if (!wait_warp(bar_k_full + 8 * ks, (kt / KS) & 1)) return false;
               tc_fence_after_sync();
             }
             issue_s(ks, hs.k0, (hs.nkeys + 15) & ~15, js & 1);
-            tc_commit(bar_s_ready + 16 * mt + 8 * (js & 1));
+            commit(bar_s_ready + 16 * mt + 8 * (js & 1));
             ++js;
             si.advance(hs);
             if (hs.last_of_tile) {
-              tc_commit(bar_k_empty + 8 * ks);
+              commit(bar_k_empty + 8 * ks);
               ++kt;
-              if (si.t >= g.t_end) tc_commit(bar_q_empty);   // Q is not read again in this segment
+              if (si.t >= g.t_end) commit(bar_q_empty);   // Q is not read again in this segment
             }
             return true;
           };
@@ -599,17 +615,17 @@ attn_step_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
           while (ok && pi.get(hs)) {
             const uint32_t vs = vt % KS;
             if (hs.first_of_tile) {
-              ok = mbar_wait(bar_v_full + 8 * vs, (vt / KS) & 1, abort_ptr);
+              ok = wait_warp(bar_v_full + 8 * vs, (vt / KS) & 1);
               if (!ok) break;
             }
-            ok = mbar_wait(bar_p_ready + 16 * mt + 8 * (gt & 1), (gt >> 1) & 1, abort_ptr);
+            ok = wait_warp(bar_p_ready + 16 * mt + 8 * (gt & 1), (gt >> 1) & 1);
             if (!ok) break;
             tc_fence_after_sync();
             issue_pv(vs, hs.k0, (hs.nkeys + 15) & ~15, gt & 1, first);
-            tc_commit(bar_pv_done + 16 * mt + 8 * (gt & 1));
+            commit(bar_pv_done + 16 * mt + 8 * (gt & 1));
             first = false;
             if (hs.last_of_tile) {
-              tc_commit(bar_v_empty + 8 * vs);
+              commit(bar_v_empty + 8 * vs);
               ++vt;
             }
             ++gt;
@@ -618,8 +634,9 @@ attn_step_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
           }
           ++seg;
         }
-        // every MMA issued by this thread has finished before TMEM is released
-        tc_commit(bar_drain + 8 * mt);
+        // every MMA issued by this warp has finished before TMEM is released
+        if (elect_one_sync()) tc_commit(bar_drain + 8 * mt);
+        __syncwarp();
         mbar_wait(bar_drain + 8 * mt, 0, &never_flag);
       }
     } else {
