@@ -138,9 +138,9 @@ size_t dlm_attn_workspace_bytes(const dlm_ctx* ctx, const dlm_kv_cache* cache,
  *   k_new, v_new device, bf16 [layers][batch][n_kv_heads][q_cap][head_dim]
  *   q_len        device, int32 [batch] or NULL (= q_cap for all)
  *   softmax_scale  <= 0 selects 1/sqrt(head_dim)
- *   cache_len_hint host upper bound on max_b cache_len[b] used only to size the launch;
- *                  <= 0 means "capacity".  A hint below the true length costs speed, not
- *                  correctness.
+ *   cache_len_hint host estimate of max_b cache_len[b], used only to choose between the two work
+ *                  schedules (units split across SMs, or dealt whole); <= 0 means "capacity".
+ *                  A poor hint costs speed, never correctness.
  *   out          device, bf16 [layers][batch][n_q_heads][q_cap][head_dim]
  *   lse          device, fp32 [layers][batch][n_q_heads][q_cap] or NULL
  *   workspace    device, 256-byte aligned, at least dlm_attn_workspace_bytes(...)

@@ -933,15 +933,28 @@ struct Plan {
   size_t ws_o_bytes, ws_ml_bytes;
 };
 
-Plan make_plan(const dlm_ctx* ctx, const dlm_kv_cache* cache, int nl, int n_q_heads, int q_cap) {
+// Splitting units across blocks balances the load perfectly but costs each block a partial
+// store and each unit a merge, about as much as kSplitCostTiles key tiles; dealing units whole
+// costs idle SMs when the units do not fill a whole number of waves.  Both are estimated from the
+// caller's cache length hint, in key tiles per block, and the cheaper one is taken.
+constexpr long long kSplitCostTiles = 5;
+
+Plan make_plan(const dlm_ctx* ctx, const dlm_kv_cache* cache, int nl, int n_q_heads, int q_cap, int cache_len_hint) {
   Plan pl;
   pl.rows = (n_q_heads / cache->n_kv_heads) * q_cap;
   pl.n_mt = (pl.rows + 127) / 128;
   const long long units = (long long)nl * cache->batch * cache->n_kv_heads;
   const int sms = ctx->num_sms < kMaxGrid ? ctx->num_sms : kMaxGrid;
-  pl.whole_units = (units >= 8LL * sms || units > kDlmMaxSplitUnits) ? 1 : 0;
+  const bool may_split = units < 8LL * sms && units <= kDlmMaxSplitUnits;
+  const int len = (cache_len_hint > 0 && cache_len_hint < cache->capacity) ? cache_len_hint : cache->capacity;
+  const long long tiles_unit = (len + 127) / 128 + (q_cap + 127) / 128;
+  const long long t_whole = ((units + sms - 1) / sms) * tiles_unit;
+  const long long t_split = (units * tiles_unit + sms - 1) / sms + kSplitCostTiles;
+  pl.whole_units = (!may_split || t_whole <= t_split) ? 1 : 0;
   pl.grid = (int)(units < sms && pl.whole_units ? units : sms);
-  const size_t slots = pl.whole_units ? 0 : 2 * (size_t)pl.grid;
+  // the workspace is sized for the split schedule whenever that schedule is possible at all, so
+  // that its size does not depend on the hint
+  const size_t slots = may_split ? 2 * (size_t)sms : 0;
   pl.ws_o_bytes = slots * pl.n_mt * 128 * cache->head_dim * sizeof(float);
   pl.ws_ml_bytes = slots * pl.n_mt * 128 * 2 * sizeof(float);
   return pl;
@@ -954,7 +967,7 @@ extern "C" size_t dlm_attn_workspace_bytes(const dlm_ctx* ctx, const dlm_kv_cach
   if (!ctx || !cache || n_layers_in_call <= 0 || n_q_heads <= 0 || q_cap <= 0 || cache->n_kv_heads <= 0 ||
       cache->batch <= 0 || n_q_heads % cache->n_kv_heads != 0)
     return 0;
-  const Plan pl = make_plan(ctx, cache, n_layers_in_call, n_q_heads, q_cap);
+  const Plan pl = make_plan(ctx, cache, n_layers_in_call, n_q_heads, q_cap, 0);
   return pl.ws_o_bytes + pl.ws_ml_bytes + 256;
 }
 
@@ -963,7 +976,6 @@ extern "C" int dlm_freecache_attn_step(dlm_ctx* ctx, const dlm_kv_cache* cache, 
                                        int q_cap, const int32_t* q_len, float softmax_scale, int cache_len_hint,
                                        void* out, float* lse, void* workspace, size_t workspace_bytes,
                                        void* stream) {
-  (void)cache_len_hint;  // the persistent schedule balances itself from the device-side lengths
   if (!ctx || !cache || !cache->k || !cache->v || !cache->cache_len || !q || !k_new || !v_new || !out)
     return DLM_ERR_NULL;
   if (cache->n_layers <= 0 || cache->batch <= 0 || cache->n_kv_heads <= 0 || cache->capacity <= 0 ||
@@ -981,7 +993,7 @@ extern "C" int dlm_freecache_attn_step(dlm_ctx* ctx, const dlm_kv_cache* cache, 
   const int nl = layer_end - layer_begin;
   const size_t need = dlm_attn_workspace_bytes(ctx, cache, nl, n_q_heads, q_cap);
   if (!workspace || workspace_bytes < need || ((uintptr_t)workspace & 255)) return DLM_ERR_WORKSPACE;
-  const Plan pl = make_plan(ctx, cache, nl, n_q_heads, q_cap);
+  const Plan pl = make_plan(ctx, cache, nl, n_q_heads, q_cap, cache_len_hint);
   {  // the split schedule counts (unit, key tile) items in 32 bits
     const long long tiles_per_unit = (cache->capacity + 127) / 128 + (q_cap + 127) / 128 + 1;
     if (!pl.whole_units && (long long)nl * cache->batch * cache->n_kv_heads * tiles_per_unit >= (1LL << 30))

@@ -57,6 +57,13 @@ def test_shapes_and_ragged_lengths(dev, oracle, Hq, Hkv, D, Lcap, q_cap, cache_l
             assert torch.all(out[:, b, :, n:] == 0)
 
 
+@pytest.mark.parametrize("hint", [1, 0])
+def test_both_schedules_whole_units_and_split(dev, oracle, hint):
+    """The length hint only picks the schedule: a tiny hint deals the units whole, the default (capacity)
+    splits these 16 long units across the SMs; both must match the oracle."""
+    _case(dev, oracle, 2, 2, 28, 4, 128, 1400, 32, [1368, 900], [32, 17], seed=77, hint=hint)
+
+
 def test_layer_range_and_explicit_scale(dev, oracle):
     _case(dev, oracle, 5, 1, 4, 2, 128, 300, 32, [290], seed=9, layer_begin=2, nl=2, scale=0.05)
 
