@@ -36,6 +36,11 @@ import torch  # noqa: E402
 from workloads import (get_config, make_attn_inputs, make_cache, make_kv_rows, make_logits,  # noqa: E402
                        seed_for, widen, bf16_bits)
 
+# dram__bytes_read.sum + dram__bytes_write.sum of one attention launch of this workload (ncu, first step of the
+# schedule: 67.06 MB read + 1.46 MB written; 73.4 MB algorithmic, most of O still being in L2 at kernel end).
+# Set to None whenever the attention kernel changes until the counters are taken again.
+ATTN_DRAM_TRAFFIC_BYTES = 68.5e6
+
 METRIC = "denoise_steps_per_s"
 UNIT = "steps/s"
 
@@ -460,7 +465,7 @@ def main():
                 "d2h_bytes_per_step": d2h, "steps": e2e_steps},
         "roofline": {"kernel": "attention step (all layers, one launch)", "bound": "hbm", "achieved": attn_gbs,
                      "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": attn_gbs / peaks["hbm_gbs"],
-                     "peak_source": peaks["source"], "traffic": None,
+                     "peak_source": peaks["source"], "traffic": ATTN_DRAM_TRAFFIC_BYTES,
                      "attn_us_per_launch": attn_ms * 1e3 / args.steps,
                      "attn_tflops": nflops / (attn_ms * 1e-3) / 1e12,
                      "algorithmic_bytes_per_launch": nbytes / args.steps},
