@@ -331,6 +331,20 @@ class Workload:
         return res
 
 
+def max_over_ranks(values, device, world):
+    """Element-wise maximum of per-rank timings over all ranks (the job runs as slow as its slowest rank)."""
+    t = torch.tensor(list(values), dtype=torch.float64, device=device)
+    if world > 1:
+        import torch.distributed as dist
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return t.tolist()
+
+
+def job_throughput(world, steps, total_ms):
+    """Whole-job steps/s: every rank runs `steps` steps of its own replica in `total_ms` (max over ranks)."""
+    return world * steps / (total_ms * 1e-3)
+
+
 def cpu_oracle_sample(cfg, cfg_index, n_layers_sample):
     """Times the CPU oracle, as it stands, on a bounded sample of one denoising step: attention for
     `n_layers_sample` of the layers at the first step's lengths, one unmask over the full block and one
@@ -446,10 +460,7 @@ def main():
     e2e_steps = min(args.steps, 64)
     e2e_ms = wl.run(e2e_steps, e2e=True, host=host)
 
-    times = torch.tensor([tot_ms, attn_ms, e2e_ms], dtype=torch.float64, device=device)
-    if world > 1:
-        dist.all_reduce(times, op=dist.ReduceOp.MAX)
-    tot_ms, attn_ms, e2e_ms = times.tolist()
+    tot_ms, attn_ms, e2e_ms = max_over_ranks([tot_ms, attn_ms, e2e_ms], device, world)
     if rank != 0:
         if world > 1:
             dist.destroy_process_group()
@@ -457,11 +468,11 @@ def main():
     peaks = measured_peaks()
     attn_gbs = nbytes / (attn_ms * 1e-3) / 1e9
     line = {
-        "metric": METRIC, "value": world * args.steps / (tot_ms * 1e-3), "unit": UNIT, "n_gpus": world,
+        "metric": METRIC, "value": job_throughput(world, args.steps, tot_ms), "unit": UNIT, "n_gpus": world,
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": tot_ms / args.steps, "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic", "config": config,
         "clocks": clocks, "gpu_launches": int(launches),
-        "e2e": {"value": world * e2e_steps / (e2e_ms * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d,
+        "e2e": {"value": job_throughput(world, e2e_steps, e2e_ms), "unit": UNIT, "h2d_bytes_per_step": h2d,
                 "d2h_bytes_per_step": d2h, "steps": e2e_steps},
         "roofline": {"kernel": "attention step (all layers, one launch)", "bound": "hbm", "achieved": attn_gbs,
                      "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": attn_gbs / peaks["hbm_gbs"],
