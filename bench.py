@@ -205,61 +205,55 @@ class Workload:
 
     def capture(self):
         """Captures the C-ABI calls of a step into CUDA graphs (the lengths and masks they read live in device
-        memory, so one capture serves every step): per input set one graph for the attention call and one for
-        unmask + commit in each of its two forms.  Replaying them removes the host's launch latency from the
+        memory, so one capture serves every step): per input set and per form of the commit, one graph holding the
+        attention call, unmask and commit, with timing events recorded inside the graph (external event nodes) before
+        the attention call, after it, and after the commit.  Replaying removes the host's launch latency from the
         device-side timing; the kernels and their arguments are exactly those of the direct calls."""
         dlm = self.dlm
         st = self.sched.at(0)
         self.reset_block_state(st)
         torch.cuda.synchronize()
-        self.g_attn, self.g_rest, self.n_attn, self.n_rest = [], [], [], []
+        self.graphs = []          # [pool index][last] -> (graph, (e0, e1, e2), kernel launches)
         side = torch.cuda.Stream()
         for i in range(self.N_POOL):
             q, kn, vn = self.pool[i]
-            g = torch.cuda.CUDAGraph()
-            c0 = dlm.dlm_launch_count(self.ctx)
-            with torch.cuda.graph(g, stream=side):
-                self.launch_attn(st, q, kn, vn)
-            self.g_attn.append(g)
-            self.n_attn.append(dlm.dlm_launch_count(self.ctx) - c0)
-            pair, counts = [], []
+            pair = []
             for last in (False, True):
+                ev = tuple(torch.cuda.Event(enable_timing=True, external=True) for _ in range(3))
                 g = torch.cuda.CUDAGraph()
                 c0 = dlm.dlm_launch_count(self.ctx)
                 with torch.cuda.graph(g, stream=side):
+                    ev[0].record()
+                    self.launch_attn(st, q, kn, vn)
+                    ev[1].record()
                     self.launch_rest(last, kn, vn, self.logits[i])
-                pair.append(g)
-                counts.append(dlm.dlm_launch_count(self.ctx) - c0)
-            self.g_rest.append(pair)
-            self.n_rest.append(counts)
+                    ev[2].record()
+                pair.append((g, ev, dlm.dlm_launch_count(self.ctx) - c0))
+            self.graphs.append(pair)
         torch.cuda.synchronize()
 
     def run_timed(self, steps):
-        """`steps` steps replayed from the graphs; L2 flushed before each; CUDA events on the launching stream
-        around the attention call and around the whole step (the flush is outside both).
-        Returns (total_ms, attn_ms, attn_bytes, attn_flops, kernel launches)."""
-        events, launches = [], 0
+        """`steps` steps replayed from the graphs; L2 flushed before each; the CUDA events inside the graph bracket
+        the attention call and the whole step on the stream the kernels run on (the flush and the graph's launch
+        latency are outside both).  Returns (total_ms, attn_ms, attn_bytes, attn_flops, kernel launches)."""
+        tot = attn = 0.0
+        launches = 0
         nbytes = nflops = 0
         for _ in range(steps):
             st = self.sched.at(self.t)
             if st["step_in_block"] == 0:
                 self.reset_block_state(st)
-            i = self.t % self.N_POOL
+            g, ev, n = self.graphs[self.t % self.N_POOL][1 if st["last"] else 0]
             self.flush.zero_()                      # evict L2 between timed steps
-            e0, e1, e2 = (torch.cuda.Event(enable_timing=True) for _ in range(3))
-            e0.record()
-            self.g_attn[i].replay()
-            e1.record()
-            self.g_rest[i][1 if st["last"] else 0].replay()
-            e2.record()
-            events.append((e0, e1, e2))
-            launches += self.n_attn[i] + self.n_rest[i][1 if st["last"] else 0]
+            g.replay()
+            ev[2].synchronize()
+            tot += ev[0].elapsed_time(ev[2])
+            attn += ev[0].elapsed_time(ev[1])
+            launches += n
             nbytes += attn_bytes(self.cfg, st["cache_len"])
             nflops += attn_flops(self.cfg, st["cache_len"])
             self.t += 1
         torch.cuda.synchronize()
-        tot = sum(a.elapsed_time(c) for a, _, c in events)
-        attn = sum(a.elapsed_time(b) for a, b, _ in events)
         return tot, attn, nbytes, nflops, launches
 
     def run(self, steps, e2e=False, host=None):
@@ -394,7 +388,7 @@ def main():
                           f"{cfg.block_len}, {cfg.steps_per_block} steps/block, vocab {cfg.vocab}, top-{cfg.top_k}",
               "attention_launch": "layer-batched (all layers in one call; synthetic stack)",
               "l2": "flushed between timed steps (512 MB write, outside the timed events)",
-              "launch": "steps replayed from CUDA graphs captured from the C-ABI calls", "parallelism": f"replicated x{world} (independent sequences)"}
+              "launch": "each step replayed from one CUDA graph captured from the C-ABI calls, timing events inside the graph", "parallelism": f"replicated x{world} (independent sequences)"}
 
     if args.impl == "reference":
         if rank != 0:
