@@ -144,8 +144,11 @@ size_t dlm_attn_workspace_bytes(const dlm_ctx* ctx, const dlm_kv_cache* cache,
  *   out          device, bf16 [layers][batch][n_q_heads][q_cap][head_dim]
  *   lse          device, fp32 [layers][batch][n_q_heads][q_cap] or NULL
  *   workspace    device, 256-byte aligned, at least dlm_attn_workspace_bytes(...)
- * Supported: head_dim in {64, 128}; n_q_heads a multiple of n_kv_heads;
- * (n_q_heads / n_kv_heads) * q_cap <= 256; q_cap >= 1.  Otherwise DLM_ERR_UNSUPPORTED.
+ * Supported: head_dim in {64, 128}; n_q_heads a multiple of n_kv_heads; 1 <= q_cap <= 4096.
+ * Otherwise DLM_ERR_UNSUPPORTED.  The (n_q_heads / n_kv_heads) * q_cap query rows that share a KV head
+ * are processed 256 at a time; each group of 256 reads that head's K/V once (the repeats normally hit L2).
+ * q_cap = the whole remaining generation is the windowed re-computation of Sec. 3.2.1; cache_len = 0 with
+ * q_cap = the whole sequence is the initial full pass that fills the cache.
  * Data-dependent: cache_len[b] outside [0, capacity] or q_len[b] outside [0, q_cap] is
  * clamped and recorded as DLM_ERR_CAPACITY; an expired device wait as DLM_ERR_TIMEOUT.
  */

@@ -46,6 +46,7 @@ constexpr int kMaxBatch = 1024;
 constexpr int kTmemCols = 512;
 constexpr int kRegsSoftmax = 216;     // registers per thread of the softmax warpgroups after setmaxnreg.inc
 constexpr int kRegsOther = 72;        // ... of the producer / MMA warpgroup after setmaxnreg.dec
+constexpr int kMaxQCap = 4096;         // active rows per call
 constexpr int kMaxGrid = 256;          // blocks of the persistent grid (one per SM)
 
 template <int D>
@@ -66,7 +67,9 @@ struct AttnParams {
   float* ws_o;    // [2 * grid][n_mt][D/4][128][4]  partial unnormalised O: 4 columns of a row per 16-byte vector
   float* ws_ml;   // [2 * grid][n_mt][128][2]    partial (running max in log2 units, running sum)
   int nl, layer_begin, batch, n_kv_heads, n_q_heads, group, capacity, q_cap;
-  int rows;        // group * q_cap: query rows per unit
+  int rows_total;  // group * q_cap: query rows per (layer, batch element, KV head)
+  int n_rc;        // row chunks: rows_total cut into units of up to 256 rows (each re-reads the K/V tiles)
+  int rows;        // query rows per unit = min(256, rows_total)
   int n_mt;        // M tiles per unit (1 or 2)
   int fresh_box;   // rows per TMA box of the fresh K/V tensors = min(128, q_cap)
   int whole_units; // 1: deal whole units round-robin, no partials
@@ -84,7 +87,7 @@ struct Sched {
 };
 
 struct Segment {
-  int lc_layer, b, kvh;   // unit
+  int lc_layer, b, kvh, rc;   // unit: layer within the call, batch element, KV head, row chunk
   int Lc, Lq, n_ct, T;    // lengths, cache tiles, total tiles of the unit
   int t_begin, t_end;     // tile range of this segment
   int slot;               // partial slot, or -1 when the segment is the whole unit
@@ -104,7 +107,7 @@ struct SegmentWalker {
   int end, range_begin;   // split mode: items [range_begin, end) are still to do
   int unit, n_units;
   __device__ SegmentWalker(const AttnParams& p_, const Sched& s_, int cta) : p(p_), s(s_) {
-    n_units = p.nl * p.n_kv_heads * p.batch;
+    n_units = p.nl * p.n_kv_heads * p.n_rc * p.batch;
     if (p.whole_units) {
       unit = cta;
       end = range_begin = 0;
@@ -119,8 +122,9 @@ struct SegmentWalker {
       if (unit >= n_units) return false;
       const int grp = unit / p.batch;
       g.b = unit % p.batch;
-      g.lc_layer = grp / p.n_kv_heads;
-      g.kvh = grp % p.n_kv_heads;
+      g.rc = grp % p.n_rc;
+      g.lc_layer = (grp / p.n_rc) / p.n_kv_heads;
+      g.kvh = (grp / p.n_rc) % p.n_kv_heads;
       g.Lc = s.lc[g.b];
       g.Lq = s.lq[g.b];
       g.T = s.prefix[g.b + 1] - s.prefix[g.b];
@@ -142,8 +146,9 @@ struct SegmentWalker {
     while (s.prefix[b + 1] <= rem) ++b;   // batch is small; units with zero tiles are skipped
     const int unit_start = grp * sum + s.prefix[b];
     g.b = b;
-    g.lc_layer = grp / p.n_kv_heads;
-    g.kvh = grp % p.n_kv_heads;
+    g.rc = grp % p.n_rc;
+    g.lc_layer = (grp / p.n_rc) / p.n_kv_heads;
+    g.kvh = (grp / p.n_rc) % p.n_kv_heads;
     g.Lc = s.lc[b];
     g.Lq = s.lq[b];
     g.T = s.prefix[b + 1] - s.prefix[b];
@@ -172,7 +177,7 @@ struct UnitPieces {
   int u0, u1, c_first, c_last;
   __device__ UnitPieces(const AttnParams& p, const Sched& s_, const Segment& g, int cta) : s(s_) {
     const int sum = s.prefix[p.batch];
-    u0 = (g.lc_layer * p.n_kv_heads + g.kvh) * sum + s.prefix[g.b];
+    u0 = ((g.lc_layer * p.n_kv_heads + g.kvh) * p.n_rc + g.rc) * sum + s.prefix[g.b];
     u1 = u0 + g.T;
     c_first = c_last = cta;
     while (s.share_lo[c_first] > u0) --c_first;
@@ -455,7 +460,7 @@ attn_step_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
   tc_fence_after_sync();
   const uint32_t tmem = tmem_slot;
   // number of shares the item list is cut into (every share holds at least one item)
-  const int total_items = sched.prefix[p.batch] * p.nl * p.n_kv_heads;
+  const int total_items = sched.prefix[p.batch] * p.nl * p.n_kv_heads * p.n_rc;
   const int n_cta = p.whole_units ? (int)gridDim.x : min((int)gridDim.x, total_items);
   const bool has_work = p.whole_units || (int)blockIdx.x < n_cta;
   if (!p.whole_units) {
@@ -488,7 +493,7 @@ attn_step_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
           for (int mt = 0; mt < p.n_mt; ++mt)
             for (int pn = 0; pn < G::kPanels; ++pn)
               tma_load_3d(sm_q + mt * G::kTileBytes + pn * kPanelBytes, &tm_q, bar_q_full, pn * 64,
-                          mt * 128, zq);
+                          g.rc * 256 + mt * 128, zq);
           for (int t = g.t_begin; t < g.t_end && ok; ++t) {
             const bool cache = t < g.n_ct;
             const int row = cache ? t * kTileKeys : (t - g.n_ct) * p.fresh_box;
@@ -653,7 +658,7 @@ attn_step_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
           if (!mbar_wait(bar_pub, pub & 1, abort_ptr)) break;
           ++pub;
           __threadfence();
-          atomicAdd(p.tickets + (g.lc_layer * p.n_kv_heads + g.kvh) * p.batch + g.b, 1u);
+          atomicAdd(p.tickets + ((g.lc_layer * p.n_kv_heads + g.kvh) * p.n_rc + g.rc) * p.batch + g.b, 1u);
         }
       }
     }
@@ -667,19 +672,19 @@ attn_step_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
       const uint32_t t_s = tmem + t_lane + G::kColS + mt * 128;
       const uint32_t t_o = tmem + t_lane + G::kColO + mt * D;
       const int r_unit = mt * 128 + row;                      // row within the unit (== tid)
-      const bool real_row = r_unit < p.rows;
-      const int h_local = real_row ? r_unit / p.q_cap : 0;
-      const int i_row = real_row ? r_unit % p.q_cap : 0;
       const int n_live_mt = min(128, n_live - 128 * mt);   // live softmax threads of this M tile
       // the warp leaves a wait together, so the .sync.aligned TMEM instructions that follow
       // always see a converged warp, also when a wait is given up
       auto wait_warp = [&](uint32_t bar, uint32_t parity) {
         return __all_sync(0xffffffffu, mbar_wait(bar, parity, abort_ptr)) != 0;
       };
-      auto out_row_of = [&](int lc_layer, int b, int kvh, int hl, int ir) {
+      // this thread's query row in row chunk rc of a KV head: which of its query heads, which active row
+      auto out_row_of = [&](int lc_layer, int b, int kvh, int rc) {
+        const int r = rc * 256 + r_unit;
+        const int hl = r < p.rows_total ? r / p.q_cap : 0, ir = r < p.rows_total ? r % p.q_cap : 0;
         return (((size_t)lc_layer * p.batch + b) * p.n_q_heads + (size_t)kvh * p.group + hl) * p.q_cap + ir;
       };
-      auto zero_my_row = [&](size_t qrow) {
+      auto zero_my_row = [&](size_t qrow, bool real_row) {
         if (real_row) {
           uint4* o = reinterpret_cast<uint4*>(p.out + qrow * D);
 #pragma unroll
@@ -689,11 +694,12 @@ attn_step_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
       };
       if (!p.whole_units) {
         // units without any key (inactive batch elements) appear in no share: zero them here
-        const int n_units = p.nl * p.n_kv_heads * p.batch;
+        const int n_units = p.nl * p.n_kv_heads * p.n_rc * p.batch;
         for (int unit = blockIdx.x; unit < n_units; unit += gridDim.x) {
-          const int b = unit % p.batch, grp = unit / p.batch;
+          const int b = unit % p.batch, grp = unit / p.batch, rc = grp % p.n_rc;
           if (sched.prefix[b + 1] == sched.prefix[b])
-            zero_my_row(out_row_of(grp / p.n_kv_heads, b, grp % p.n_kv_heads, h_local, i_row));
+            zero_my_row(out_row_of((grp / p.n_rc) / p.n_kv_heads, b, (grp / p.n_rc) % p.n_kv_heads, rc),
+                        rc * 256 + r_unit < p.rows_total);
         }
       }
       if (has_work) {
@@ -703,9 +709,12 @@ attn_step_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
         bool ok = true;
         while (ok && walk.next(g, n_cta)) {
           const int n = g.t_end - g.t_begin;
-          const size_t qrow = out_row_of(g.lc_layer, g.b, g.kvh, h_local, i_row);
+          const size_t qrow = out_row_of(g.lc_layer, g.b, g.kvh, g.rc);
+          const int r_kv = g.rc * 256 + r_unit;               // row among all query rows of the KV head
+          const bool real_row = r_kv < p.rows_total;
+          const int i_row = real_row ? r_kv % p.q_cap : 0;
           if (n <= 0) {  // whole-unit mode, inactive batch element: the unit's rows are zero
-            zero_my_row(qrow);
+            zero_my_row(qrow, real_row);
             continue;
           }
           float m_used = -CUDART_INF_F, l_run = 0.f;
@@ -806,7 +815,7 @@ attn_step_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
               // them into O (own piece first, then block order: the result does not depend on timing).
               const UnitPieces up(p, sched, g, blockIdx.x);
               const int n_others = up.c_last - up.c_first;
-              const int unit = (g.lc_layer * p.n_kv_heads + g.kvh) * p.batch + g.b;
+              const int unit = ((g.lc_layer * p.n_kv_heads + g.kvh) * p.n_rc + g.rc) * p.batch + g.b;
               if (tid == 0) {
                 merge_ok = wait_counter(p.tickets + unit, (unsigned int)n_others, abort_ptr) ? 1 : 0;
                 if (merge_ok) p.tickets[unit] = 0;   // ready for the next launch
@@ -929,7 +938,7 @@ bool register_budget_ok(const void* kern) {
 }
 
 struct Plan {
-  int n_mt, rows, grid, whole_units;
+  int n_mt, rows, rows_total, n_rc, grid, whole_units;
   size_t ws_o_bytes, ws_ml_bytes;
 };
 
@@ -941,9 +950,11 @@ constexpr long long kSplitCostTiles = 5;
 
 Plan make_plan(const dlm_ctx* ctx, const dlm_kv_cache* cache, int nl, int n_q_heads, int q_cap, int cache_len_hint) {
   Plan pl;
-  pl.rows = (n_q_heads / cache->n_kv_heads) * q_cap;
+  pl.rows_total = (n_q_heads / cache->n_kv_heads) * q_cap;
+  pl.n_rc = (pl.rows_total + 255) / 256;
+  pl.rows = pl.rows_total < 256 ? pl.rows_total : 256;
   pl.n_mt = (pl.rows + 127) / 128;
-  const long long units = (long long)nl * cache->batch * cache->n_kv_heads;
+  const long long units = (long long)nl * cache->batch * cache->n_kv_heads * pl.n_rc;
   const int sms = ctx->num_sms < kMaxGrid ? ctx->num_sms : kMaxGrid;
   const bool may_split = units < 8LL * sms && units <= kDlmMaxSplitUnits;
   const int len = (cache_len_hint > 0 && cache_len_hint < cache->capacity) ? cache_len_hint : cache->capacity;
@@ -986,7 +997,7 @@ extern "C" int dlm_freecache_attn_step(dlm_ctx* ctx, const dlm_kv_cache* cache, 
   if (D != 64 && D != 128) return DLM_ERR_UNSUPPORTED;
   if (n_q_heads % cache->n_kv_heads != 0) return DLM_ERR_UNSUPPORTED;
   const int group = n_q_heads / cache->n_kv_heads;
-  if ((long long)group * q_cap > 256 || cache->batch > kMaxBatch) return DLM_ERR_UNSUPPORTED;
+  if (q_cap > kMaxQCap || (long long)group * q_cap > (1 << 20) || cache->batch > kMaxBatch) return DLM_ERR_UNSUPPORTED;
   if (((uintptr_t)cache->k | (uintptr_t)cache->v | (uintptr_t)q | (uintptr_t)k_new | (uintptr_t)v_new |
        (uintptr_t)out) & 15)
     return DLM_ERR_UNSUPPORTED;
@@ -996,7 +1007,7 @@ extern "C" int dlm_freecache_attn_step(dlm_ctx* ctx, const dlm_kv_cache* cache, 
   const Plan pl = make_plan(ctx, cache, nl, n_q_heads, q_cap, cache_len_hint);
   {  // the split schedule counts (unit, key tile) items in 32 bits
     const long long tiles_per_unit = (cache->capacity + 127) / 128 + (q_cap + 127) / 128 + 1;
-    if (!pl.whole_units && (long long)nl * cache->batch * cache->n_kv_heads * tiles_per_unit >= (1LL << 30))
+    if (!pl.whole_units && (long long)nl * cache->batch * cache->n_kv_heads * pl.n_rc * tiles_per_unit >= (1LL << 30))
       return DLM_ERR_UNSUPPORTED;
   }
 
@@ -1016,6 +1027,8 @@ extern "C" int dlm_freecache_attn_step(dlm_ctx* ctx, const dlm_kv_cache* cache, 
   p.capacity = cache->capacity;
   p.q_cap = q_cap;
   p.rows = pl.rows;
+  p.rows_total = pl.rows_total;
+  p.n_rc = pl.n_rc;
   p.n_mt = pl.n_mt;
   p.fresh_box = q_cap < 128 ? q_cap : 128;
   p.whole_units = pl.whole_units;
@@ -1028,7 +1041,7 @@ extern "C" int dlm_freecache_attn_step(dlm_ctx* ctx, const dlm_kv_cache* cache, 
   const long long slabs_new = (long long)nl * cache->batch * cache->n_kv_heads;
   const long long slabs_cache = (long long)cache->n_layers * cache->batch * cache->n_kv_heads;
   const int cache_box = cache->capacity < 128 ? cache->capacity : 128;
-  int rc = encode_map(ctx, &tm_q, q, D, pl.rows, slabs_new, pl.rows < 128 ? pl.rows : 128);
+  int rc = encode_map(ctx, &tm_q, q, D, pl.rows_total, slabs_new, pl.rows < 128 ? pl.rows : 128);
   if (rc == DLM_OK) rc = encode_map(ctx, &tm_kc, cache->k, D, cache->capacity, slabs_cache, cache_box);
   if (rc == DLM_OK) rc = encode_map(ctx, &tm_vc, cache->v, D, cache->capacity, slabs_cache, cache_box);
   if (rc == DLM_OK) rc = encode_map(ctx, &tm_kn, k_new, D, q_cap, slabs_new, p.fresh_box);

@@ -64,6 +64,20 @@ def test_both_schedules_whole_units_and_split(dev, oracle, hint):
     _case(dev, oracle, 2, 2, 28, 4, 128, 1400, 32, [1368, 900], [32, 17], seed=77, hint=hint)
 
 
+@pytest.mark.parametrize("Hq,Hkv,D,Lcap,q_cap,cache_len,q_len", [
+    (28, 4, 128, 600, 256, [300], None),                # the paper's window: 256 active rows, Dream heads (7 chunks of 256 rows)
+    (4, 4, 128, 520, 512, [0, 0], [512, 333]),          # initial full pass: empty cache, 512 active rows, ragged
+    (4, 2, 64, 400, 300, [77, 100], [300, 130]),        # rows per KV head not a multiple of 256, head_dim 64
+])
+def test_large_windows_in_row_chunks(dev, oracle, Hq, Hkv, D, Lcap, q_cap, cache_len, q_len):
+    B = len(cache_len)
+    for hint in (1, 0):   # both schedules
+        out, lse, _ = _case(dev, oracle, 1, B, Hq, Hkv, D, Lcap, q_cap, cache_len, q_len, seed=Hq * 1000 + q_cap, hint=hint)
+        if q_len is not None:
+            for b, n in enumerate(q_len):
+                assert torch.all(out[:, b, :, n:] == 0)
+
+
 def test_layer_range_and_explicit_scale(dev, oracle):
     _case(dev, oracle, 5, 1, 4, 2, 128, 300, 32, [290], seed=9, layer_begin=2, nl=2, scale=0.05)
 
@@ -107,7 +121,7 @@ def test_argument_errors(dev):
                                     torch.empty_like(q), None, ws_)
 
     before = dlm.dlm_launch_count(dev.ctx)
-    for kwargs, code in ((dict(Hq=3), dlm.DLM_ERR_UNSUPPORTED), (dict(Hq=4, q_cap=200), dlm.DLM_ERR_UNSUPPORTED),
+    for kwargs, code in ((dict(Hq=3), dlm.DLM_ERR_UNSUPPORTED), (dict(Hq=4, q_cap=5000), dlm.DLM_ERR_UNSUPPORTED),
                          (dict(layer_end=2), dlm.DLM_ERR_SHAPE),
                          (dict(ws_=ws[8:]), dlm.DLM_ERR_WORKSPACE)):
         with pytest.raises(dlm.DlmError) as e:
