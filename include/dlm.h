@@ -235,6 +235,22 @@ int dlm_guided_accept(dlm_ctx* ctx, const int32_t* tok_dlm, const int32_t* tok_a
                       int block_len, uint8_t* masked, int32_t* tokens, int fallback_source,
                       uint8_t* accept, int32_t* acc_idx, int32_t* n_acc, void* stream);
 
+/*
+ * dlm_guided_accept_topk — the "Top-K Match" variant of the accept rule (App. C.1, Table 7: Top-1 / Top-2 /
+ * Top-5 match; App. C.3 configuration table: "Top-K Assisted Tokens Selection", default 2).
+ *
+ * As dlm_guided_accept, except that position i counts as agreeing when tok_dlm[i] equals ANY of the
+ * guider's top_k tokens for position i.  The paper names the variant without a formula; this is the reading
+ * taken.  top_k = 1 is dlm_guided_accept.
+ *
+ *   tok_ar_topk  device, int32 [batch][block_len][top_k], the guider's tokens for each position in rank
+ *                order (entry 0 is its argmax, which is also the AR token of fallback_source == 1)
+ * Supported: block_len <= 1024, 1 <= top_k <= 64.
+ */
+int dlm_guided_accept_topk(dlm_ctx* ctx, const int32_t* tok_dlm, const int32_t* tok_ar_topk, int top_k, int batch,
+                           int block_len, uint8_t* masked, int32_t* tokens, int fallback_source,
+                           uint8_t* accept, int32_t* acc_idx, int32_t* n_acc, void* stream);
+
 #ifdef __cplusplus
 }
 #endif

@@ -119,3 +119,19 @@ def guided_accept(tok_dlm, tok_ar, masked, tokens, fallback_source=0):
         _p(acc_idx, np.int32), _p(n_acc, np.int32))
     assert rc == 0, rc
     return accept, acc_idx, n_acc
+
+
+def guided_accept_topk(tok_dlm, tok_ar_topk, masked, tokens, fallback_source=0):
+    """Top-K match variant: tok_ar_topk int32 [B,Lblk,K] in rank order.  Returns (accept, acc_idx, n_acc)."""
+    B, Lblk = tok_dlm.shape
+    K = tok_ar_topk.shape[2]
+    assert tok_ar_topk.shape == (B, Lblk, K)
+    accept = np.empty((B, Lblk), np.uint8)
+    acc_idx = np.empty((B, Lblk), np.int32)
+    n_acc = np.empty((B,), np.int32)
+    rc = _load().oracle_guided_accept_topk(
+        B, Lblk, K, _p(tok_dlm, np.int32), _p(tok_ar_topk, np.int32), _p(masked, np.uint8),
+        _p(tokens, np.int32), int(fallback_source), _p(accept, np.uint8),
+        _p(acc_idx, np.int32), _p(n_acc, np.int32))
+    assert rc == 0, rc
+    return accept, acc_idx, n_acc

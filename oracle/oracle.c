@@ -276,3 +276,48 @@ int oracle_guided_accept(int B, int Lblk, const int32_t* tok_dlm, const int32_t*
   }
   return ORACLE_OK;
 }
+
+/*
+ * "Top-K Match" variant of the accept rule (App. C.1, Table 7; configuration table of App. C.3).
+ * The paper names it without a formula; the reading taken: position i_j agrees when tok_dlm[i_j] equals any
+ * of the guider's K tokens for that position.  Everything else is the rule above: longest agreeing prefix
+ * over the masked positions in ascending order, the first masked position alone if it does not agree.
+ * tok_ar_topk is [B][Lblk][K] in rank order; entry 0 is the guider's argmax (the AR fallback token).
+ */
+int oracle_guided_accept_topk(int B, int Lblk, int K, const int32_t* tok_dlm, const int32_t* tok_ar_topk,
+                              uint8_t* masked, int32_t* tokens, int fallback_source,
+                              uint8_t* accept, int32_t* acc_idx, int32_t* n_acc) {
+  if (K <= 0) return -1;
+  for (int b = 0; b < B; ++b) {
+    const size_t o = (size_t)b * Lblk;
+    int n = 0, first = -1, still_agreeing = 1;
+    for (int i = 0; i < Lblk; ++i) { accept[o + i] = 0; acc_idx[o + i] = -1; }
+    for (int i = 0; i < Lblk; ++i) {
+      if (!masked[o + i]) continue;
+      if (first < 0) first = i;
+      if (!still_agreeing) continue;
+      int among = 0;
+      for (int j = 0; j < K; ++j)
+        if (tok_ar_topk[(o + i) * K + j] == tok_dlm[o + i]) among = 1;
+      if (among) {
+        accept[o + i] = 1;
+        acc_idx[o + n++] = i;
+      } else {
+        still_agreeing = 0;
+      }
+    }
+    int fallback = 0;
+    if (n == 0 && first >= 0) {
+      accept[o + first] = 1;
+      acc_idx[o + n++] = first;
+      fallback = 1;
+    }
+    for (int j = 0; j < n; ++j) {
+      const int i = acc_idx[o + j];
+      tokens[o + i] = (fallback && fallback_source == 1) ? tok_ar_topk[(o + i) * K] : tok_dlm[o + i];
+      masked[o + i] = 0;
+    }
+    n_acc[b] = n;
+  }
+  return ORACLE_OK;
+}

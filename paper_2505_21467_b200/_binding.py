@@ -64,8 +64,9 @@ def lib() -> ctypes.CDLL:
     L.dlm_unmask_select.argtypes = [vp, vp, i32, i32, i32, vp, vp, i32, vp, vp, vp, vp, vp, sz, vp]
     L.dlm_unmask_select_static.argtypes = [vp, i32, i32, i32, vp, vp, i32, vp, vp, vp, vp, vp]
     L.dlm_guided_accept.argtypes = [vp, vp, vp, i32, i32, vp, vp, i32, vp, vp, vp, vp]
+    L.dlm_guided_accept_topk.argtypes = [vp, vp, vp, i32, i32, i32, vp, vp, i32, vp, vp, vp, vp]
     for name in ("dlm_create", "dlm_destroy", "dlm_get_status", "dlm_kv_cache_commit",
-                 "dlm_freecache_attn_step", "dlm_unmask_select", "dlm_unmask_select_static", "dlm_guided_accept"):
+                 "dlm_freecache_attn_step", "dlm_unmask_select", "dlm_unmask_select_static", "dlm_guided_accept", "dlm_guided_accept_topk"):
         getattr(L, name).restype = i32
     _lib = L
     return L
@@ -175,3 +176,11 @@ def dlm_guided_accept(ctx, tok_dlm, tok_ar, batch, block_len, masked, tokens, fa
         ctx, _ptr(tok_dlm, torch.int32), _ptr(tok_ar, torch.int32), int(batch), int(block_len),
         _ptr(masked, torch.uint8), _ptr(tokens, torch.int32), int(fallback_source), _ptr(accept, torch.uint8),
         _ptr(acc_idx, torch.int32), _ptr(n_acc, torch.int32), _stream()), "dlm_guided_accept")
+
+
+def dlm_guided_accept_topk(ctx, tok_dlm, tok_ar_topk, top_k, batch, block_len, masked, tokens, fallback_source, accept,
+                           acc_idx, n_acc) -> None:
+    _check(lib().dlm_guided_accept_topk(
+        ctx, _ptr(tok_dlm, torch.int32), _ptr(tok_ar_topk, torch.int32), int(top_k), int(batch), int(block_len),
+        _ptr(masked, torch.uint8), _ptr(tokens, torch.int32), int(fallback_source), _ptr(accept, torch.uint8),
+        _ptr(acc_idx, torch.int32), _ptr(n_acc, torch.int32), _stream()), "dlm_guided_accept_topk")

@@ -8,7 +8,7 @@
 namespace {
 
 __global__ void __launch_bounds__(32)
-guided_accept_kernel(const int32_t* __restrict__ tok_dlm, const int32_t* __restrict__ tok_ar, int block_len,
+guided_accept_kernel(const int32_t* __restrict__ tok_dlm, const int32_t* __restrict__ tok_ar, int top_k, int block_len,
                      uint8_t* __restrict__ masked, int32_t* __restrict__ tokens, int fallback_source,
                      uint8_t* __restrict__ accept, int32_t* __restrict__ acc_idx, int32_t* __restrict__ n_acc) {
   const int b = blockIdx.x;
@@ -23,7 +23,12 @@ guided_accept_kernel(const int32_t* __restrict__ tok_dlm, const int32_t* __restr
     const bool in = i < block_len;
     const bool m = in && masked[o + i] != 0;
     const int td = in ? tok_dlm[o + i] : 0;
-    const bool agree = m && td == tok_ar[in ? o + i : o];
+    // agreement: the DLM token is among the guider's top_k tokens for this position (top_k = 1: its argmax)
+    bool agree = false;
+    if (m) {
+      const int32_t* cand = tok_ar + (o + i) * top_k;
+      for (int j = 0; j < top_k; ++j) agree = agree || cand[j] == td;
+    }
     const unsigned mm = __ballot_sync(0xffffffffu, m);
     const unsigned dis = __ballot_sync(0xffffffffu, m && !agree);
     if (first_masked < 0 && mm) first_masked = base + __ffs(mm) - 1;
@@ -48,7 +53,7 @@ guided_accept_kernel(const int32_t* __restrict__ tok_dlm, const int32_t* __restr
       const size_t q = o + first_masked;
       accept[q] = 1;
       acc_idx[o] = first_masked;
-      tokens[q] = fallback_source == 1 ? tok_ar[q] : tok_dlm[q];
+      tokens[q] = fallback_source == 1 ? tok_ar[q * top_k] : tok_dlm[q];
       masked[q] = 0;
     }
     n = 1;
@@ -66,6 +71,17 @@ extern "C" int dlm_guided_accept(dlm_ctx* ctx, const int32_t* tok_dlm, const int
   if (batch <= 0 || block_len <= 0) return DLM_ERR_SHAPE;
   if (block_len > 1024 || (fallback_source != 0 && fallback_source != 1)) return DLM_ERR_UNSUPPORTED;
   guided_accept_kernel<<<batch, 32, 0, static_cast<cudaStream_t>(stream)>>>(
-      tok_dlm, tok_ar, block_len, masked, tokens, fallback_source, accept, acc_idx, n_acc);
+      tok_dlm, tok_ar, 1, block_len, masked, tokens, fallback_source, accept, acc_idx, n_acc);
+  return dlm_launch_ok(ctx, 1);
+}
+
+extern "C" int dlm_guided_accept_topk(dlm_ctx* ctx, const int32_t* tok_dlm, const int32_t* tok_ar_topk, int top_k,
+                                      int batch, int block_len, uint8_t* masked, int32_t* tokens, int fallback_source,
+                                      uint8_t* accept, int32_t* acc_idx, int32_t* n_acc, void* stream) {
+  if (!ctx || !tok_dlm || !tok_ar_topk || !masked || !tokens || !accept || !acc_idx || !n_acc) return DLM_ERR_NULL;
+  if (batch <= 0 || block_len <= 0 || top_k <= 0) return DLM_ERR_SHAPE;
+  if (block_len > 1024 || top_k > 64 || (fallback_source != 0 && fallback_source != 1)) return DLM_ERR_UNSUPPORTED;
+  guided_accept_kernel<<<batch, 32, 0, static_cast<cudaStream_t>(stream)>>>(
+      tok_dlm, tok_ar_topk, top_k, block_len, masked, tokens, fallback_source, accept, acc_idx, n_acc);
   return dlm_launch_ok(ctx, 1);
 }

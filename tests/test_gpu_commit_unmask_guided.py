@@ -301,3 +301,31 @@ def test_guided_config_statistics(dev, oracle):
     a = make_tok_ar(torch.from_numpy(d), cfg.p_agree, cfg.vocab, 2).numpy()
     n = _compare_guided(dev, oracle, d, a, np.ones((B, Lblk), np.uint8))
     assert abs(n.mean() - (0.2 + 4 * (1 - 0.8 ** 32))) < 0.25
+
+
+@pytest.mark.parametrize("K", [1, 2, 5])
+def test_guided_topk_match_variant(dev, oracle, K):
+    """Top-K match: bit-exact against the oracle on random blocks with a small vocabulary (agreements at every
+    rank are common), both fallback sources, block lengths on both sides of a warp."""
+    rng = np.random.default_rng(40 + K)
+    for Lblk in (7, 32, 70):
+        B, V = 64, 6
+        d = rng.integers(0, V, (B, Lblk)).astype(np.int32)
+        a = np.stack([rng.permutation(V)[:K] for _ in range(B * Lblk)]).reshape(B, Lblk, K).astype(np.int32)
+        masked0 = (rng.random((B, Lblk)) < 0.6).astype(np.uint8)
+        for source in (0, 1):
+            o_m, o_t = masked0.copy(), np.full((B, Lblk), -1, np.int32)
+            o_acc, o_idx, o_n = oracle.guided_accept_topk(d, a, o_m, o_t, source)
+            g_m = torch.from_numpy(masked0.copy()).cuda()
+            g_t = torch.full((B, Lblk), -1, dtype=torch.int32, device="cuda")
+            accept = torch.empty(B, Lblk, dtype=torch.uint8, device="cuda")
+            acc_idx = torch.empty(B, Lblk, dtype=torch.int32, device="cuda")
+            n_acc = torch.empty(B, dtype=torch.int32, device="cuda")
+            dlm.dlm_guided_accept_topk(dev.ctx, torch.from_numpy(d).cuda(), torch.from_numpy(a).cuda(), K, B, Lblk, g_m, g_t,
+                                       source, accept, acc_idx, n_acc)
+            np.testing.assert_array_equal(accept.cpu().numpy(), o_acc)
+            np.testing.assert_array_equal(acc_idx.cpu().numpy(), o_idx)
+            np.testing.assert_array_equal(n_acc.cpu().numpy(), o_n)
+            np.testing.assert_array_equal(g_m.cpu().numpy(), o_m)
+            np.testing.assert_array_equal(g_t.cpu().numpy(), o_t)
+    assert dev.status() == 0

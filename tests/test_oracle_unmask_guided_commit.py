@@ -255,6 +255,64 @@ def test_guided_exhaustive_agreement_patterns(oracle, m):
         np.testing.assert_array_equal(tokens[b, pos[:want]], dlm[b, pos[:want]])
 
 
+def test_guided_topk_handworked_fixture(oracle):
+    for line in open(os.path.join(GOLDEN, "guided_accept_topk_handworked.txt")):
+        if not line.strip() or line.startswith("#"):
+            continue
+        f = line.rstrip("\n").split("|")
+        masked0 = np.array(f[0].split(), np.int64)
+        dlm = np.array(f[1].split(), np.int32)
+        ar = np.array([[int(t) for t in pair.split(",")] for pair in f[2].split()], np.int32)
+        want, w0, w1 = (np.array(x.split(), np.int64) for x in f[3:6])
+        for source, written in ((0, w0), (1, w1)):
+            masked = masked0.astype(np.uint8)[None].copy()
+            tokens = np.full(masked.shape, -5, np.int32)
+            accept, acc_idx, n_acc = oracle.guided_accept_topk(dlm[None], ar[None], masked, tokens, source)
+            assert n_acc[0] == len(want)
+            np.testing.assert_array_equal(acc_idx[0, :len(want)], want)
+            assert np.all(acc_idx[0, len(want):] == -1)
+            exp_tokens = np.full(len(masked0), -5, np.int32)
+            exp_tokens[want] = written
+            np.testing.assert_array_equal(tokens[0], exp_tokens)
+            exp_accept = np.zeros(len(masked0), np.uint8)
+            exp_accept[want] = 1
+            np.testing.assert_array_equal(accept[0], exp_accept)
+            np.testing.assert_array_equal(masked[0], masked0.astype(np.uint8) & (1 - exp_accept))
+
+
+@pytest.mark.parametrize("K", [1, 2, 5])
+def test_guided_topk_against_set_membership_brute_force(oracle, K):
+    """Random small blocks against a plain Python statement of the rule with sets; K = 1 must also equal the
+    Top-1 rule (itself pinned by the exhaustive test above)."""
+    rng = np.random.default_rng(100 + K)
+    B, Lblk, V = 300, 9, 6                                  # tiny vocabulary: agreements at every rank are common
+    dlm = rng.integers(0, V, (B, Lblk)).astype(np.int32)
+    ar = np.stack([rng.permutation(V)[:K] for _ in range(B * Lblk)]).reshape(B, Lblk, K).astype(np.int32)
+    masked0 = (rng.random((B, Lblk)) < 0.7).astype(np.uint8)
+    for source in (0, 1):
+        masked, tokens = masked0.copy(), np.full((B, Lblk), -1, np.int32)
+        accept, acc_idx, n_acc = oracle.guided_accept_topk(dlm, ar, masked, tokens, source)
+        for b in range(B):
+            M = [i for i in range(Lblk) if masked0[b, i]]
+            lead = 0
+            while lead < len(M) and int(dlm[b, M[lead]]) in set(ar[b, M[lead]].tolist()):
+                lead += 1
+            want = M[:max(lead, 1)] if M else []
+            assert n_acc[b] == len(want) and list(acc_idx[b, :len(want)]) == want
+            for i in range(Lblk):
+                if i in want:
+                    exp = ar[b, i, 0] if (lead == 0 and source == 1) else dlm[b, i]
+                    assert tokens[b, i] == exp and masked[b, i] == 0 and accept[b, i] == 1
+                else:
+                    assert tokens[b, i] == -1 and masked[b, i] == masked0[b, i] and accept[b, i] == 0
+        if K == 1:
+            m1, t1 = masked0.copy(), np.full((B, Lblk), -1, np.int32)
+            a1, i1, n1 = oracle.guided_accept(dlm, ar[:, :, 0].copy(), m1, t1, source)
+            np.testing.assert_array_equal(a1, accept)
+            np.testing.assert_array_equal(i1, acc_idx)
+            np.testing.assert_array_equal(t1, tokens)
+
+
 def test_commit_window_mode_stages_rows_at_their_own_slots(oracle):
     """dst_mode 1: fresh row p goes to slot cache_len + p, whatever its place in the index list."""
     ck, cv, kn, vn = _commit_case(500)
