@@ -72,6 +72,12 @@ const char* dlm_strerror(int code);
 /* Number of kernels this context has launched so far (host-side counter). */
 int64_t dlm_launch_count(const dlm_ctx* ctx);
 
+/* Diagnostic: enqueues a one-warp kernel that waits, with the library's bounded device-side wait and a
+ * limit of `limit_ns` nanoseconds (1 .. 1e9), on a barrier nobody arrives at.  The wait gives up, the
+ * kernel ends normally and dlm_get_status then reports DLM_ERR_TIMEOUT; the context stays usable.  This is
+ * how the give-up path of every wait in the kernels is exercised without hanging a GPU. */
+int dlm_selftest_wait_timeout(dlm_ctx* ctx, uint64_t limit_ns, void* stream);
+
 /* View of a caller-owned KV cache (Sec. 3.2.1: K/V of the prompt and of frozen blocks).
  *   k, v       device, bf16 [n_layers][batch][n_kv_heads][capacity][head_dim]
  *   cache_len  device, int32 [batch]: rows [0, cache_len[b]) are visible to attention.

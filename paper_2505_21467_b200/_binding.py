@@ -51,6 +51,8 @@ def lib() -> ctypes.CDLL:
     L.dlm_get_status.argtypes = [vp, vp]
     L.dlm_strerror.argtypes = [i32]
     L.dlm_strerror.restype = ctypes.c_char_p
+    L.dlm_selftest_wait_timeout.argtypes = [vp, ctypes.c_uint64, vp]
+    L.dlm_selftest_wait_timeout.restype = i32
     L.dlm_launch_count.argtypes = [vp]
     L.dlm_launch_count.restype = ctypes.c_int64
     L.dlm_kv_cache_commit.argtypes = [vp, ctypes.POINTER(dlm_kv_cache), vp, vp, i32, vp, vp, i32, vp, i32, i32,
@@ -184,3 +186,7 @@ def dlm_guided_accept_topk(ctx, tok_dlm, tok_ar_topk, top_k, batch, block_len, m
         ctx, _ptr(tok_dlm, torch.int32), _ptr(tok_ar_topk, torch.int32), int(top_k), int(batch), int(block_len),
         _ptr(masked, torch.uint8), _ptr(tokens, torch.int32), int(fallback_source), _ptr(accept, torch.uint8),
         _ptr(acc_idx, torch.int32), _ptr(n_acc, torch.int32), _stream()), "dlm_guided_accept_topk")
+
+
+def dlm_selftest_wait_timeout(ctx, limit_ns: int) -> None:
+    _check(lib().dlm_selftest_wait_timeout(ctx, ctypes.c_uint64(int(limit_ns)), _stream()), "dlm_selftest_wait_timeout")

@@ -2,6 +2,7 @@
 #include <new>
 
 #include "common.cuh"
+#include "sm100_ptx.cuh"
 
 extern "C" int dlm_create(dlm_ctx** out, int device) {
   if (!out) return DLM_ERR_NULL;
@@ -68,4 +69,27 @@ extern "C" const char* dlm_strerror(int code) {
     case DLM_ERR_INDEX: return "a row index is out of range";
     default: return "unknown error code";
   }
+}
+
+namespace {
+
+// Waits on an mbarrier that nobody will ever arrive at, with the same bounded wait the kernels use.
+__global__ void wait_probe_kernel(unsigned long long limit_ns, int* status) {
+  __shared__ uint64_t bar;
+  __shared__ int abort_flag;
+  if (threadIdx.x == 0) {
+    abort_flag = 0;
+    sm100::mbar_init(sm100::smem_u32(&bar), 1);
+    sm100::mbar_fence_init();
+    if (!sm100::mbar_wait_limit(sm100::smem_u32(&bar), 0, &abort_flag, limit_ns)) dlm_set_status(status, DLM_ERR_TIMEOUT);
+  }
+}
+
+}  // namespace
+
+extern "C" int dlm_selftest_wait_timeout(dlm_ctx* ctx, uint64_t limit_ns, void* stream) {
+  if (!ctx) return DLM_ERR_NULL;
+  if (limit_ns == 0 || limit_ns > 1000000000ull) return DLM_ERR_SHAPE;   // at most one second
+  wait_probe_kernel<<<1, 32, 0, static_cast<cudaStream_t>(stream)>>>(limit_ns, &ctx->words->status);
+  return dlm_launch_ok(ctx, 1);
 }

@@ -176,3 +176,15 @@ def test_llada_shape_sampled(dev, oracle):
     cfg = get_config(2)
     _case(dev, oracle, 2, cfg.batch, cfg.n_q_heads, cfg.n_kv_heads, cfg.head_dim, cfg.capacity, cfg.block_len,
           [2048, 2112, 2496, 2300], seed=seed_for(2), layers=[1], device="cuda")
+
+
+def test_a_wait_that_runs_out_reports_timeout_and_leaves_the_context_usable(dev, oracle):
+    """The bounded device-side wait gives up after its limit (here 2 ms on a barrier nothing arrives at): the kernel
+    ends normally, the status word says DLM_ERR_TIMEOUT, it is cleared by the read, and the next calls work."""
+    dlm.dlm_selftest_wait_timeout(dev.ctx, 2_000_000)
+    assert dev.status() == dlm.DLM_ERR_TIMEOUT
+    assert dev.status() == 0
+    _case(dev, oracle, 1, 1, 4, 2, 64, 200, 16, [150], seed=5)
+    with pytest.raises(dlm.DlmError) as e:
+        dlm.dlm_selftest_wait_timeout(dev.ctx, 5_000_000_000)
+    assert e.value.code == dlm.DLM_ERR_SHAPE
