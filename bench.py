@@ -118,14 +118,17 @@ class Schedule:
 
     def __init__(self, cfg):
         self.cfg = cfg
-        self.n = cfg.n_blocks * cfg.steps_per_block
+        # guided policy: the number of steps a block takes depends on the data; the schedule gives it 8
+        # (about 4.2 positions are accepted per step of a 32-position block) and then moves on
+        self.steps_per_block = cfg.steps_per_block if cfg.policy == "topk" else 8
+        self.n = cfg.n_blocks * self.steps_per_block
 
     def at(self, t):
         cfg = self.cfg
         t %= self.n
-        block, s = divmod(t, cfg.steps_per_block)
+        block, s = divmod(t, self.steps_per_block)
         return {"block": block, "step_in_block": s, "cache_len": cfg.prompt_len + block * cfg.block_len,
-                "n_masked": cfg.block_len - s * cfg.top_k, "last": s == cfg.steps_per_block - 1}
+                "n_masked": cfg.block_len - s * cfg.top_k, "last": s == self.steps_per_block - 1}
 
 
 def attn_bytes(cfg, cache_len):
@@ -163,30 +166,61 @@ class Workload:
         self.tokens = torch.full((B, Lblk), -1, dtype=torch.int32, device=device)
         self.tok = torch.empty(B, Lblk, dtype=torch.int32, device=device)
         self.conf = torch.empty(B, Lblk, dtype=torch.float32, device=device)
-        self.sel_idx = torch.empty(B, cfg.top_k, dtype=torch.int32, device=device)
+        self.sel_idx = torch.empty(B, max(cfg.top_k, 1), dtype=torch.int32, device=device)
         self.n_sel = torch.empty(B, dtype=torch.int32, device=device)
         self.attn_ws = torch.empty(max(dlm.dlm_attn_workspace_bytes(self.ctx, self.cache, cfg.n_layers, cfg.n_q_heads,
                                                                     Lblk), 256), dtype=torch.uint8, device=device)
         self.unmask_ws = torch.empty(max(dlm.dlm_unmask_workspace_bytes(self.ctx, B, Lblk, V), 256),
                                      dtype=torch.uint8, device=device)
         self.flush = torch.empty(512 << 20, dtype=torch.uint8, device=device)   # 4x the 126 MB L2
+        self.guided = cfg.policy == "guided"
+        if self.guided:
+            # the guider's argmax for every position: agrees with the DLM's argmax with probability p_agree
+            self.q_len = torch.full((B,), Lblk, dtype=torch.int32, device=device)
+            self.accept = torch.empty(B, Lblk, dtype=torch.uint8, device=device)
+            self.acc_idx = torch.empty(B, Lblk, dtype=torch.int32, device=device)
+            self.n_acc = torch.empty(B, dtype=torch.int32, device=device)
+            self.tok_ar = []
+            from workloads import make_tok_ar
+            for i in range(self.N_POOL):
+                self.masked.fill_(1)
+                dlm.dlm_unmask_select(self.ctx, self.logits[i], B, Lblk, V, self.masked, self.tokens, 0, self.tok, self.conf,
+                                      None, None, self.unmask_ws)
+                self.tok_ar.append(make_tok_ar(self.tok.cpu(), cfg.p_agree, V, s + 20 + i).to(device))
         self.sched = Schedule(cfg)
         self.t = 0
 
     def reset_block_state(self, st):
         """Puts the device state where step `t` of the schedule expects it (not timed)."""
         self.cache_len.fill_(st["cache_len"])
+        if self.guided:     # accepted positions form a prefix: a block starts fully masked
+            if st["step_in_block"] == 0:
+                self.masked.fill_(1)
+            self.q_len.copy_(self.masked.sum(1))
+            return
         self.masked.zero_()
         self.masked[:, :st["n_masked"]] = 1
 
     def launch_attn(self, st, q, kn, vn):
         dlm, cfg = self.dlm, self.cfg
         dlm.dlm_freecache_attn_step(self.ctx, self.cache, 0, cfg.n_layers, q, kn, vn, cfg.n_q_heads, cfg.block_len,
-                                    None, 0.0, st["cache_len"], self.out, None, self.attn_ws)
+                                    self.q_len if self.guided else None, 0.0, st["cache_len"], self.out, None, self.attn_ws)
 
     def launch_rest(self, last, kn, vn, lg):
         """Unmask, then the commit: the 4 staged rows, or the whole block when it completes."""
         dlm, cfg = self.dlm, self.cfg
+        if self.guided:
+            # propose (argmax for every masked position), accept the prefix the guider agrees with, append the
+            # accepted rows (visible at once); the window shrinks to the still-masked rows
+            i = 0 if lg is self.logits[0] else 1
+            dlm.dlm_unmask_select(self.ctx, lg, cfg.batch, cfg.block_len, cfg.vocab, self.masked, self.tokens, 0,
+                                  self.tok, self.conf, None, None, self.unmask_ws)
+            dlm.dlm_guided_accept(self.ctx, self.tok, self.tok_ar[i], cfg.batch, cfg.block_len, self.masked, self.tokens, 0,
+                                  self.accept, self.acc_idx, self.n_acc)
+            dlm.dlm_kv_cache_commit(self.ctx, self.cache, kn, vn, cfg.block_len, self.acc_idx, None, dlm.DLM_DST_APPEND,
+                                    self.n_acc, cfg.block_len, 1, 0, cfg.n_layers)
+            self.q_len.copy_(self.masked.sum(1))
+            return
         dlm.dlm_unmask_select(self.ctx, lg, cfg.batch, cfg.block_len, cfg.vocab, self.masked, self.tokens, cfg.top_k,
                               self.tok, self.conf, self.sel_idx, self.n_sel, self.unmask_ws)
         if last:      # block complete: freeze all of its rows and make them visible
@@ -355,18 +389,32 @@ def cpu_oracle_sample(cfg, cfg_index, n_layers_sample):
     t_attn = (time.perf_counter() - t0) / n_layers_sample
     logits = make_logits(B, Lblk, cfg.vocab, cfg.logit_sigma, s + 10).numpy()
     masked, tokens = np.ones((B, Lblk), np.uint8), np.zeros((B, Lblk), np.int32)
-    t0 = time.perf_counter()
-    _, _, sel, n = oracle.unmask_select(logits, masked, tokens, cfg.top_k)
-    t_unmask = time.perf_counter() - t0
     cks, cvs = bf16_bits(ck), bf16_bits(cv)
     knb, vnb = bf16_bits(kn), bf16_bits(vn)
-    t0 = time.perf_counter()
-    oracle.kv_cache_commit(cks, cvs, np.full((B,), cfg.prompt_len, np.int32), knb, vnb, sel, None, n, cfg.top_k, dst_mode=1)
-    t_commit = (time.perf_counter() - t0) * cfg.n_layers
+    lens = np.full((B,), cfg.prompt_len, np.int32)
+    if cfg.policy == "guided":
+        from workloads import make_tok_ar
+        t0 = time.perf_counter()
+        tok, _, _, _ = oracle.unmask_select(logits, masked, tokens, 0)
+        tok_ar = make_tok_ar(torch.from_numpy(tok), cfg.p_agree, cfg.vocab, s + 20).numpy()
+        _, idx, n = oracle.guided_accept(tok, tok_ar, masked, tokens, 0)
+        t_unmask = time.perf_counter() - t0
+        t0 = time.perf_counter()
+        oracle.kv_cache_commit(cks, cvs, lens, knb, vnb, idx, None, n, Lblk, True)
+        t_commit = (time.perf_counter() - t0) * cfg.n_layers
+        what = "one propose + guided accept"
+    else:
+        t0 = time.perf_counter()
+        _, _, sel, n = oracle.unmask_select(logits, masked, tokens, cfg.top_k)
+        t_unmask = time.perf_counter() - t0
+        t0 = time.perf_counter()
+        oracle.kv_cache_commit(cks, cvs, lens, knb, vnb, sel, None, n, cfg.top_k, dst_mode=1)
+        t_commit = (time.perf_counter() - t0) * cfg.n_layers
+        what = "one unmask"
     step_s = cfg.n_layers * t_attn + t_unmask + t_commit
     return {"value": 1.0 / step_s, "unit": UNIT, "cores": oracle.num_threads(), "kind": "oracle",
             "sample": f"attention of {n_layers_sample} of {cfg.n_layers} layers at cache_len {cfg.prompt_len} "
-                      f"(x{cfg.n_layers}/{n_layers_sample}), one unmask over {Lblk}x{cfg.vocab} logits, one 4-row commit",
+                      f"(x{cfg.n_layers}/{n_layers_sample}), {what} over {B}x{Lblk}x{cfg.vocab} logits, one commit of the chosen rows",
             "seconds_per_step": step_s}
 
 
@@ -383,7 +431,7 @@ def main():
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
-    config = {"workload": f"{cfg.name}: Dream-7B-shaped attention stack, batch {cfg.batch} per GPU, {cfg.n_layers} layers, "
+    config = {"workload": f"{cfg.name}: {'LLaDA-8B' if cfg.name == 'llada8b' else 'Dream-7B'}-shaped attention stack, batch {cfg.batch} per GPU, {cfg.n_layers} layers, "
                           f"{cfg.n_q_heads}q/{cfg.n_kv_heads}kv heads x {cfg.head_dim}, prompt {cfg.prompt_len} + {cfg.n_blocks} blocks of "
                           f"{cfg.block_len}, {cfg.steps_per_block} steps/block, vocab {cfg.vocab}, top-{cfg.top_k}",
               "attention_launch": "layer-batched (all layers in one call; synthetic stack)",
@@ -475,7 +523,7 @@ def main():
                      "attn_tflops": nflops / (attn_ms * 1e-3) / 1e12,
                      "algorithmic_bytes_per_launch": nbytes / args.steps},
         "other_kernels": wl.other_kernels(peaks["hbm_gbs"]),
-        "cpu_baseline": cpu_oracle_sample(cfg, cfg_index, 4),
+        "cpu_baseline": cpu_oracle_sample(cfg, cfg_index, max(1, min(4, int(2.5e9 / max(attn_flops(cfg, cfg.prompt_len) / cfg.n_layers, 1))))),
     }
     print(json.dumps(line))
     if world > 1:
