@@ -327,6 +327,30 @@ class Workload:
         ts = sorted(a.elapsed_time(b) for a, b in evs)
         return ts[len(ts) // 2] * 1e-3
 
+    def per_layer_attention(self):
+        """The attention of one step issued the way a real model would: one call per layer, here all in one graph,
+        at the first step's lengths (the headline number uses the layer-batched call, which only a synthetic stack,
+        whose layers' Q/K/V all exist up front, can make)."""
+        dlm, cfg = self.dlm, self.cfg
+        st = self.sched.at(0)
+        self.reset_block_state(st)
+        q, kn, vn = self.pool[0]
+        ws = torch.empty(max(dlm.dlm_attn_workspace_bytes(self.ctx, self.cache, 1, cfg.n_q_heads, cfg.block_len), 256),
+                         dtype=torch.uint8, device=self.dev)
+
+        def layers():
+            for l in range(cfg.n_layers):
+                dlm.dlm_freecache_attn_step(self.ctx, self.cache, l, l + 1, q[l:l + 1], kn[l:l + 1], vn[l:l + 1], cfg.n_q_heads,
+                                            cfg.block_len, self.q_len if self.guided else None, 0.0, st["cache_len"],
+                                            self.out[l:l + 1], None, ws)
+        layers()
+        torch.cuda.synchronize()
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g, stream=torch.cuda.Stream()):
+            layers()
+        t = self.time_call(g.replay)
+        return {"us_per_step": t * 1e6, "us_per_layer": t * 1e6 / cfg.n_layers, "calls": cfg.n_layers}
+
     def other_kernels(self, peak_gbs):
         """HBM-bound kernels of the path, each timed alone from a captured graph: the unmask pass over a fully
         masked block and the cache refresh that (re)writes the whole prompt."""
@@ -526,6 +550,7 @@ def main():
                      "attn_tflops": nflops / (attn_ms * 1e-3) / 1e12,
                      "algorithmic_bytes_per_launch": nbytes / args.steps},
         "other_kernels": wl.other_kernels(peaks["hbm_gbs"]),
+        "attention_per_layer_calls": wl.per_layer_attention(),
         "cpu_baseline": cpu_oracle_sample(cfg, cfg_index, max(1, min(4, int(2.5e9 / max(attn_flops(cfg, cfg.prompt_len) / cfg.n_layers, 1))))),
     }
     print(json.dumps(line))
