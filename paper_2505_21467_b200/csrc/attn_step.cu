@@ -268,16 +268,16 @@ __device__ __noinline__ bool rescale_o(uint32_t t_o, bool grow, float m_new, flo
   return true;
 }
 
-// Full half-step (64 valid keys): the score row sits in registers between the maximum and the
-// exponentials, so TMEM is read once and with a single wait.
+// Full half-step (64 valid keys): the score row sits in registers, so TMEM is read once and with a
+// single wait.  Only the first half-step of a segment takes the row maximum before the
+// exponentials; later ones form P against the maximum in use and look at the row sum afterwards:
+// a sum above kSumLimit means some score outgrew that maximum by a lot, and only then (rare)
+// is the maximum taken, O rescaled and P formed again.  The maximum pass, half-rate ALU work
+// that both softmax groups of an SMSP would do at the same time, is gone from the steady state.
+constexpr float kSumLimit = 1024.0f;   // 64 keys: some P is then above 16, and none was above 1024 before
+
 template <int D>
-__device__ __forceinline__ bool softmax_half_full(uint32_t t_s, uint32_t t_o, bool first, float scale_log2,
-                                                  float& m_used, float& l_run, uint32_t bar_pv_done,
-                                                  uint32_t pv_parity, volatile int* abort_ptr) {
-  uint32_t s[64];
-  tmem_ld32(t_s, s);
-  tmem_ld32(t_s + 32, s + 32);
-  tmem_ld_wait();
+__device__ __forceinline__ float row_max64(const uint32_t (&s)[64]) {
   float mx[8];   // independent chains: the maximum is latency-bound otherwise
 #pragma unroll
   for (int c = 0; c < 8; ++c) mx[c] = __uint_as_float(s[c]);
@@ -286,17 +286,12 @@ __device__ __forceinline__ bool softmax_half_full(uint32_t t_s, uint32_t t_o, bo
 #pragma unroll
     for (int c = 0; c < 8; ++c) mx[c] = fmaxf(mx[c], __uint_as_float(s[j + c]));
   }
-  const float m_new =
-      fmaxf(fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3])), fmaxf(fmaxf(mx[4], mx[5]), fmaxf(mx[6], mx[7]))) * scale_log2;
-  if (first) {
-    m_used = m_new;
-    l_run = 0.f;
-  } else {
-    const bool grow = m_new > m_used + kRescaleThreshold;
-    if (__any_sync(0xffffffffu, grow)) {
-      if (!rescale_o<D>(t_o, grow, m_new, m_used, l_run, bar_pv_done, pv_parity, abort_ptr)) return false;
-    }
-  }
+  return fmaxf(fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3])), fmaxf(fmaxf(mx[4], mx[5]), fmaxf(mx[6], mx[7])));
+}
+
+// P = 2^(s * scale - m) for the 64 scores, packed to bf16 pairs and written over the scores in TMEM;
+// returns the row sum.
+__device__ __forceinline__ float exp64_store(const uint32_t (&s)[64], float scale_log2, float m_used, uint32_t t_s) {
   float l0 = 0.f, l1 = 0.f;
 #pragma unroll
   for (int c = 0; c < 2; ++c) {
@@ -312,7 +307,32 @@ __device__ __forceinline__ bool softmax_half_full(uint32_t t_s, uint32_t t_o, bo
     }
     tmem_st16(t_s + c * 16, pk);
   }
-  l_run += l0 + l1;
+  return l0 + l1;
+}
+
+template <int D>
+__device__ __forceinline__ bool softmax_half_full(uint32_t t_s, uint32_t t_o, bool first, float scale_log2,
+                                                  float& m_used, float& l_run, uint32_t bar_pv_done,
+                                                  uint32_t pv_parity, volatile int* abort_ptr) {
+  uint32_t s[64];
+  tmem_ld32(t_s, s);
+  tmem_ld32(t_s + 32, s + 32);
+  tmem_ld_wait();
+  if (first) {
+    m_used = row_max64<D>(s) * scale_log2;
+    l_run = 0.f;
+  }
+  float l_half = exp64_store(s, scale_log2, m_used, t_s);
+  if (!first) {
+    const bool grow = !(l_half <= kSumLimit);   // also catches a NaN sum
+    if (__any_sync(0xffffffffu, grow)) {
+      const float m_new = row_max64<D>(s) * scale_log2;
+      tmem_st_wait();   // the P just written is replaced below
+      if (!rescale_o<D>(t_o, grow, m_new, m_used, l_run, bar_pv_done, pv_parity, abort_ptr)) return false;
+      l_half = exp64_store(s, scale_log2, m_used, t_s);
+    }
+  }
+  l_run += l_half;
   tmem_st_wait();
   return true;
 }

@@ -78,6 +78,24 @@ def test_large_windows_in_row_chunks(dev, oracle, Hq, Hkv, D, Lcap, q_cap, cache
                 assert torch.all(out[:, b, :, n:] == 0)
 
 
+@pytest.mark.parametrize("scale", [0.2, 1.0])
+def test_scores_that_keep_outgrowing_the_running_maximum(dev, oracle, scale):
+    """Keys grow along the cache and the softmax scale is large, so later tiles bring scores far above the
+    maximum in use (by tens of powers of two): the deferred rescaling of O has to fire, repeatedly, and the result
+    must still match.  Both schedules."""
+    NL, B, Hq, Hkv, D, Lc, q_cap = 1, 2, 14, 2, 128, 1500, 32
+    ck, cv = make_cache(NL, B, Hkv, Lc + 40, D, 91)
+    q, kn, vn = make_attn_inputs(NL, B, Hq, Hkv, q_cap, D, 92)
+    grow = (1.0 + 4.0 * torch.arange(Lc + 40, dtype=torch.float32) / Lc).view(1, 1, 1, -1, 1)
+    ck = (ck.float() * grow).to(torch.bfloat16)
+    cl = _i32([Lc, Lc - 333])
+    for hint in (1, 0):
+        out, lse = gpu_attn_step(dev, ck.cuda(), cv.cuda(), cl, q.cuda(), kn.cuda(), vn.cuda(), None, scale, hint=hint)
+        assert dev.status() == 0
+        ref = oracle_attn_layers(oracle, ck, cv, cl, q, kn, vn, None, scale)
+        assert_attn_close(out, lse, ref[0], 0)
+
+
 def test_layer_range_and_explicit_scale(dev, oracle):
     _case(dev, oracle, 5, 1, 4, 2, 128, 300, 32, [290], seed=9, layer_begin=2, nl=2, scale=0.05)
 
