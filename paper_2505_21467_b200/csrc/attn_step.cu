@@ -738,47 +738,44 @@ attn_step_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
             continue;
           }
           float m_used = -CUDART_INF_F, l_run = 0.f;
-          HalfIter hi(g, p.fresh_box);
-          HalfStep hs;
           bool first = true;
-          while (ok && hi.get(hs)) {
-            if (hs.first_of_tile) {
-              const int valid = tile_valid(g, hs.t, p.fresh_box);
-              const int n16 = (valid + 15) & ~15;
-              if (valid < n16) {
-                // V rows in [valid, n16) would be multiplied by P = 0: clear them so that stale
-                // NaN / Inf bit patterns cannot reach O.  Each M tile's warps do it before they
-                // announce the P of the tile's first half-step, so it precedes that tile's P V
-                // products (the two M tiles write the same zeros).
-                const uint32_t vs = vt % KS;
-                ok = wait_warp(bar_v_full + 8 * vs, (vt / KS) & 1);
-                if (!ok) break;
-                const int per_row = G::kPanels * 8;
-                for (int idx = row; idx < (n16 - valid) * per_row; idx += n_live_mt) {
-                  const int r = valid + idx / per_row, rem = idx % per_row;
-                  const uint32_t a = sm_v + vs * G::kTileBytes + (rem >> 3) * kPanelBytes + r * 128 + (rem & 7) * 16;
-                  asm volatile("st.shared.v4.b32 [%0], {%1, %1, %1, %1};" ::"r"(a), "r"(0u) : "memory");
-                }
-                fence_proxy_async_smem();
+          for (int t = g.t_begin; t < g.t_end && ok; ++t, ++vt) {
+            const int valid = tile_valid(g, t, p.fresh_box);
+            const int n16 = (valid + 15) & ~15;
+            if (valid < n16) {
+              // V rows in [valid, n16) would be multiplied by P = 0: clear them so that stale
+              // NaN / Inf bit patterns cannot reach O.  Each M tile's warps do it before they
+              // announce the P of the tile's first half-step, so it precedes that tile's P V
+              // products (the two M tiles write the same zeros).
+              const uint32_t vs = vt % KS;
+              ok = wait_warp(bar_v_full + 8 * vs, (vt / KS) & 1);
+              if (!ok) break;
+              const int per_row = G::kPanels * 8;
+              for (int idx = row; idx < (n16 - valid) * per_row; idx += n_live_mt) {
+                const int r = valid + idx / per_row, rem = idx % per_row;
+                const uint32_t a = sm_v + vs * G::kTileBytes + (rem >> 3) * kPanelBytes + r * 128 + (rem & 7) * 16;
+                asm volatile("st.shared.v4.b32 [%0], {%1, %1, %1, %1};" ::"r"(a), "r"(0u) : "memory");
               }
+              fence_proxy_async_smem();
             }
-            const uint32_t buf = gt & 1;
-            ok = wait_warp(bar_s_ready + 16 * mt + 8 * buf, (gt >> 1) & 1);
-            if (!ok) break;
-            tc_fence_after_sync();
-            if (hs.nkeys == kHalfKeys)
-              ok = softmax_half_full<D>(t_s + buf * kHalfKeys, t_o, first, p.scale_log2, m_used, l_run,
-                                        bar_pv_done + 16 * mt + 8 * ((gt - 1) & 1), ((gt - 1) >> 1) & 1, abort_ptr);
-            else
-              ok = softmax_half_ragged<D>(t_s + buf * kHalfKeys, t_o, hs.nkeys, first, p.scale_log2, m_used, l_run,
+            // the tile's half-steps (the same enumeration as HalfIter, which the MMA warps use)
+            for (int k0 = 0; k0 < valid && ok; k0 += kHalfKeys, ++gt) {
+              const int nkeys = min(kHalfKeys, valid - k0);
+              const uint32_t buf = gt & 1;
+              ok = wait_warp(bar_s_ready + 16 * mt + 8 * buf, (gt >> 1) & 1);
+              if (!ok) break;
+              tc_fence_after_sync();
+              if (nkeys == kHalfKeys)
+                ok = softmax_half_full<D>(t_s + buf * kHalfKeys, t_o, first, p.scale_log2, m_used, l_run,
                                           bar_pv_done + 16 * mt + 8 * ((gt - 1) & 1), ((gt - 1) >> 1) & 1, abort_ptr);
-            if (!ok) break;
-            tc_fence_before_sync();
-            mbar_arrive(bar_p_ready + 16 * mt + 8 * buf);
-            first = false;
-            ++gt;
-            if (hs.last_of_tile) ++vt;
-            hi.advance(hs);
+              else
+                ok = softmax_half_ragged<D>(t_s + buf * kHalfKeys, t_o, nkeys, first, p.scale_log2, m_used, l_run,
+                                            bar_pv_done + 16 * mt + 8 * ((gt - 1) & 1), ((gt - 1) >> 1) & 1, abort_ptr);
+              if (!ok) break;
+              tc_fence_before_sync();
+              mbar_arrive(bar_p_ready + 16 * mt + 8 * buf);
+              first = false;
+            }
           }
           if (!ok) break;
           // ---- epilogue of the segment: O is complete once the last P V product has finished
