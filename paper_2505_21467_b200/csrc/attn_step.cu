@@ -420,27 +420,10 @@ attn_step_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
   // softmax threads that own a real query row, rounded up to whole warps (they are tid 0 .. n_live-1)
   const int n_live = (p.rows + 31) & ~31;
 
-  // ---- set-up: lengths and tile prefix, barriers, TMEM
-  if (tid == 0) { abort_flag = 0; never_flag = 0; merge_ok = 0; }
-  for (int b = tid; b < p.batch; b += kThreads) {
-    int Lc = p.cache_len[b];
-    int Lq = p.q_len ? p.q_len[b] : p.q_cap;
-    if (Lc < 0 || Lc > p.capacity || Lq < 0 || Lq > p.q_cap) {
-      dlm_set_status(p.status, DLM_ERR_CAPACITY);
-      Lc = max(0, min(Lc, p.capacity));
-      Lq = max(0, min(Lq, p.q_cap));
-    }
-    sched.lc[b] = Lc;
-    sched.lq[b] = Lq;
-  }
-  __syncthreads();
+  // ---- set-up: barriers, TMEM and descriptor prefetch first (they need no data), so that they overlap
+  // the cold read of the lengths; then the tile prefix
   if (tid == 0) {
-    int acc = 0;
-    for (int b = 0; b < p.batch; ++b) {
-      sched.prefix[b] = acc;
-      acc += tiles_of(sched.lc[b], sched.lq[b], p.fresh_box);
-    }
-    sched.prefix[p.batch] = acc;
+    abort_flag = 0; never_flag = 0; merge_ok = 0;
     mbar_init(bar_q_full, 1);
     mbar_init(bar_q_empty, (uint32_t)p.n_mt);       // one commit per MMA issuer
     mbar_init(bar_drain, 1);
@@ -474,6 +457,26 @@ attn_step_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
     prefetch_tensormap(&tm_vc);
     prefetch_tensormap(&tm_kn);
     prefetch_tensormap(&tm_vn);
+  }
+  for (int b = tid; b < p.batch; b += kThreads) {
+    int Lc = p.cache_len[b];
+    int Lq = p.q_len ? p.q_len[b] : p.q_cap;
+    if (Lc < 0 || Lc > p.capacity || Lq < 0 || Lq > p.q_cap) {
+      dlm_set_status(p.status, DLM_ERR_CAPACITY);
+      Lc = max(0, min(Lc, p.capacity));
+      Lq = max(0, min(Lq, p.q_cap));
+    }
+    sched.lc[b] = Lc;
+    sched.lq[b] = Lq;
+  }
+  __syncthreads();
+  if (tid == 0) {
+    int acc = 0;
+    for (int b = 0; b < p.batch; ++b) {
+      sched.prefix[b] = acc;
+      acc += tiles_of(sched.lc[b], sched.lq[b], p.fresh_box);
+    }
+    sched.prefix[p.batch] = acc;
   }
   tc_fence_before_sync();
   __syncthreads();
