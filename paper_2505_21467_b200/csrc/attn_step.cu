@@ -962,12 +962,12 @@ struct Plan {
   size_t ws_o_bytes, ws_ml_bytes;
 };
 
-// Splitting units across blocks balances the load perfectly but costs each block a partial
-// store and each unit a merge, about as much as kSplitCostTiles key tiles; dealing units whole
-// costs idle SMs when the units do not fill a whole number of waves.  Both are estimated from the
-// caller's cache length hint, in key tiles per block, and the cheaper one is taken.
-constexpr long long kSplitCostTiles = 5;
-
+// Splitting units across blocks balances the load but costs each block a partial store and each
+// unit a wait and a merge that grows with its number of pieces (measured: about 3 key tiles' worth
+// plus 0.7 per further piece); dealing units whole costs idle SMs when the units do not fill a
+// whole number of waves.  The number of shares (= blocks) is chosen to minimise the estimated
+// time in key tiles per block, from the caller's cache length hint; one share per unit or fewer
+// means whole units.
 Plan make_plan(const dlm_ctx* ctx, const dlm_kv_cache* cache, int nl, int n_q_heads, int q_cap, int cache_len_hint) {
   Plan pl;
   pl.rows_total = (n_q_heads / cache->n_kv_heads) * q_cap;
@@ -979,10 +979,23 @@ Plan make_plan(const dlm_ctx* ctx, const dlm_kv_cache* cache, int nl, int n_q_he
   const bool may_split = units < 8LL * sms && units <= kDlmMaxSplitUnits;
   const int len = (cache_len_hint > 0 && cache_len_hint < cache->capacity) ? cache_len_hint : cache->capacity;
   const long long tiles_unit = (len + 127) / 128 + (q_cap + 127) / 128;
-  const long long t_whole = ((units + sms - 1) / sms) * tiles_unit;
-  const long long t_split = (units * tiles_unit + sms - 1) / sms + kSplitCostTiles;
-  pl.whole_units = (!may_split || t_whole <= t_split) ? 1 : 0;
-  pl.grid = (int)(units < sms && pl.whole_units ? units : sms);
+  const double t_whole = (double)(((units + sms - 1) / sms) * tiles_unit);
+  double best = t_whole;
+  int best_shares = 0;   // 0: whole units
+  if (may_split) {
+    for (long long shares = units + 1; shares <= sms; ++shares) {
+      if (shares > units * tiles_unit) break;   // a share holds at least one item
+      const double pieces = (double)shares / (double)units;
+      const double t = (double)((units * tiles_unit + shares - 1) / shares) + 3.0 + 0.7 * (pieces - 1.0);
+      if (t < best) { best = t; best_shares = (int)shares; }
+    }
+    if (units > sms) {   // more units than SMs: the only split is over all SMs
+      const double t = (double)((units * tiles_unit + sms - 1) / sms) + 3.0 + 0.7;
+      if (t < best) { best = t; best_shares = sms; }
+    }
+  }
+  pl.whole_units = best_shares == 0 ? 1 : 0;
+  pl.grid = pl.whole_units ? (int)(units < sms ? units : sms) : best_shares;
   // the workspace is sized for the split schedule whenever that schedule is possible at all, so
   // that its size does not depend on the hint
   const size_t slots = may_split ? 2 * (size_t)sms : 0;
