@@ -2,22 +2,24 @@
 // (Sec. 3.2.1 "Windowed Re-computation"; Table 1 rows QK^T and Attention Score x Value;
 // bidirectional: no causal mask).
 //
-// One work unit is (layer, batch element, KV head): all g = Hq/Hkv query heads of that KV
-// head, q_cap rows each, form up to two 128-row M tiles that share every K/V tile, so K/V are
-// read from HBM once per KV head.  Keys are visited in tiles of 128 rows: first the visible
-// cache rows, then the fresh rows.
+// One work unit is (layer, batch element, KV head, chunk of up to 256 query rows): the g = Hq/Hkv
+// query heads of a KV head, q_cap rows each, are cut into chunks of 256 rows = two 128-row M
+// tiles that share every K/V tile (at the block sizes of the configs, g * q_cap <= 256: one chunk,
+// K/V read from HBM once per KV head; larger windows re-read them per chunk, normally from L2).
+// Keys are loaded in tiles of 128 rows, first the visible cache rows, then the fresh rows, and
+// processed in half-steps of 64.
 //
 // Block = 12 warps (three warpgroups), one block per SM (persistent):
 //   warps 0-3   softmax of M tile 0 (thread = query row = TMEM lane)
 //   warps 4-7   softmax of M tile 1
 //   warp  8     TMA producer (one lane): Q once per segment, K and V tiles through two rings
-//   warp  9/10  tcgen05.mma issuer of M tile 0 / 1 (one lane each): S = Q K^T into TMEM, then
+//   warp  9/10  tcgen05.mma issuer of M tile 0 / 1 (one elected lane each): S = Q K^T into one of two
+//               64-column score buffers in TMEM, two half-steps ahead of the softmax; then
 //               O += P V with P read from TMEM (it overwrites S in place as packed bf16)
 //   warp  11    publisher (one lane): makes a finished partial result visible device-wide and
 //               bumps its unit's counter, so the softmax warps need not wait for that
-// Online softmax in fp32 with base-2 exponentials; a whole score row sits in registers between
-// the maximum and the exponentials; O stays in TMEM and is rescaled only when a row maximum has
-// grown by more than a threshold.
+// Online softmax in fp32 with base-2 exponentials; a half-step's scores sit in registers; O stays
+// in TMEM and is rescaled only when a row's scores have outgrown the maximum in use by a lot.
 //
 // Scheduling.  Every (unit, key tile) pair is one item of a global list; block c takes the
 // contiguous share [c*T/G, (c+1)*T/G) of it.  A share covers whole units (result written
@@ -26,8 +28,8 @@
 // share (the last piece of its unit) is the last thing the block computes; that block merges the
 // unit: it waits for the counter the other pieces' blocks bump after publishing their partial
 // results (they have lower block indices and computed those pieces first), then folds them into
-// its own O, which is still in TMEM, in block order: the result is deterministic.  With many
-// more units than SMs the split is not worth its traffic and units are dealt round-robin instead.
+// its own O, which is still in TMEM, in block order: the result is deterministic.  When the split
+// would cost more than it saves (the host estimates both) units are dealt whole, round-robin.
 #include <cuda.h>
 #include <cuda_bf16.h>
 #include <math_constants.h>
@@ -237,10 +239,11 @@ struct HalfIter {
 };
 
 // Softmax of one half-step for the query row held by this thread (S row in TMEM -> P row in TMEM).
-// O is rescaled only when the running maximum has grown by more than kRescaleThreshold (log2
-// units): until then P is formed against the older, smaller maximum and may reach
-// 2^kRescaleThreshold, which bf16 and the fp32 accumulators hold just as well; the final division
-// by the row sum, taken against the same maximum, cancels it.
+// O is rescaled only when the scores have outgrown the maximum in use by a lot: until then P is
+// formed against the older, smaller maximum and may exceed 1 by a few powers of two, which bf16
+// and the fp32 accumulators hold just as well; the final division by the row sum, taken against
+// the same maximum, cancels it.  Ragged half-steps compare maxima (kRescaleThreshold, log2 units);
+// full ones look at the row sum (kSumLimit).
 constexpr float kRescaleThreshold = 8.0f;
 
 // Rare path shared by both kinds of half-step: some row of the warp outgrew its maximum by more
