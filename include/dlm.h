@@ -17,8 +17,8 @@
  *     argument error is returned nothing has been launched.
  *   - Pointers documented "device" are caller-owned device pointers on the context's GPU and
  *     must stay valid until the enqueued work has finished.  The library never allocates,
- *     frees or retains tensor memory; the only device memory it owns is a few hundred bytes
- *     of status and ticket words inside the context.
+ *     frees or retains tensor memory; the only device memory it owns is about 12 KB of
+ *     status and ticket words inside the context.
  *   - `stream` is a cudaStream_t passed as void* (NULL = the default stream).  All calls
  *     only enqueue work; none synchronises except dlm_get_status.
  *   - Data-dependent errors (an index out of range, an append beyond capacity, a bounded
