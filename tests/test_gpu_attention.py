@@ -182,6 +182,16 @@ def test_guided_shape_ragged_batch8(dev, oracle):
           cache_len, q_len, seed=seed_for(4), layers=[0, 2])
 
 
+def test_guided_shape_more_units_than_sms_split_schedule(dev, oracle):
+    """Config 5's launch form: more units (10 layers x 8 sequences x 4 KV heads = 320) than SMs and still split,
+    so a block's share holds whole units and a partial unit at each end, with ragged lengths."""
+    cfg = get_config(4)
+    cache_len = [1024, 1031, 1056, 1100, 1247, 1279, 1088, 1150]
+    q_len = [32, 25, 32, 20, 1, 1, 32, 2]
+    _case(dev, oracle, 10, cfg.batch, cfg.n_q_heads, cfg.n_kv_heads, cfg.head_dim, cfg.capacity, cfg.block_len,
+          cache_len, q_len, seed=seed_for(4, 7), layers=[0, 9], device="cuda")
+
+
 def test_longctx_shape_sampled_layers(dev, oracle):
     """Config 4: 16384 cached rows, Dream heads; 4 of the 28 layers resident, oracle on two of them."""
     cfg = get_config(3)
