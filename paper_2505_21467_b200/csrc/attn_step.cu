@@ -461,6 +461,9 @@ attn_step_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
     prefetch_tensormap(&tm_kn);
     prefetch_tensormap(&tm_vn);
   }
+  // everything above needed no data; from here on the inputs of the call are read
+  dlm_grid_dependency_wait();
+  dlm_trigger_dependents();
   for (int b = tid; b < p.batch; b += kThreads) {
     int Lc = p.cache_len[b];
     int Lq = p.q_len ? p.q_len[b] : p.q_cap;
@@ -1093,7 +1096,7 @@ extern "C" int dlm_freecache_attn_step(dlm_ctx* ctx, const dlm_kv_cache* cache, 
       DLM_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, Geometry<128>::kSmemBytes));
       configured = true;
     }
-    kern<<<pl.grid, kThreads, Geometry<128>::kSmemBytes, s>>>(tm_q, tm_kc, tm_vc, tm_kn, tm_vn, p);
+    DLM_CUDA_TRY(dlm_launch(kern, dim3(pl.grid), dim3(kThreads), Geometry<128>::kSmemBytes, s, tm_q, tm_kc, tm_vc, tm_kn, tm_vn, p));
   } else {
     auto kern = attn_step_sm100_kernel<64>;
     static bool configured = false;
@@ -1102,7 +1105,7 @@ extern "C" int dlm_freecache_attn_step(dlm_ctx* ctx, const dlm_kv_cache* cache, 
       DLM_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, Geometry<64>::kSmemBytes));
       configured = true;
     }
-    kern<<<pl.grid, kThreads, Geometry<64>::kSmemBytes, s>>>(tm_q, tm_kc, tm_vc, tm_kn, tm_vn, p);
+    DLM_CUDA_TRY(dlm_launch(kern, dim3(pl.grid), dim3(kThreads), Geometry<64>::kSmemBytes, s, tm_q, tm_kc, tm_vc, tm_kn, tm_vn, p));
   }
   return dlm_launch_ok(ctx, 1);
 }

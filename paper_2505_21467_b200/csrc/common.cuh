@@ -37,6 +37,34 @@ struct dlm_ctx {
 // Records the first error seen by any thread of any kernel.
 __device__ __forceinline__ void dlm_set_status(int* status, int code) { atomicCAS(status, 0, code); }
 
+// Programmatic dependent launch.  Every kernel of the library is launched with the
+// programmatic-stream-serialization attribute, calls dlm_grid_dependency_wait() before it touches
+// anything a predecessor in the stream may have written, and lets its own dependents start
+// launching early with dlm_trigger_dependents(): block scheduling and the dependents' data-free
+// set-up then overlap the predecessor's tail instead of following it.  A dependent's wait still
+// returns only when the predecessor grid has completed and its writes are visible, and the
+// hardware starts dependents only once every block of the predecessor is running, so nothing is
+// reordered.  Predecessors that know nothing of this (any other kernel) simply release their
+// dependents when they finish.
+__device__ __forceinline__ void dlm_grid_dependency_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void dlm_trigger_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
+template <typename... KArgs, typename... Args>
+static inline cudaError_t dlm_launch(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t stream,
+                                     Args... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid;
+  cfg.blockDim = block;
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = stream;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+}
+
 static inline int dlm_launch_ok(dlm_ctx* ctx, int n_kernels) {
   if (cudaGetLastError() != cudaSuccess) return DLM_ERR_CUDA;
   ctx->launches += n_kernels;

@@ -41,6 +41,8 @@ __device__ __forceinline__ int valid_rows(const CommitParams& p, int b, int len0
 }
 
 __global__ void __launch_bounds__(kThreads) kv_commit_kernel(const CommitParams p) {
+  dlm_grid_dependency_wait();
+  dlm_trigger_dependents();
   const long long stride = (long long)gridDim.x * kThreads;
   const long long first = (long long)blockIdx.x * kThreads + threadIdx.x;
   for (long long base = first; base < p.n_items; base += stride * kUnroll) {
@@ -161,6 +163,6 @@ extern "C" int dlm_kv_cache_commit(dlm_ctx* ctx, const dlm_kv_cache* cache, cons
   const long long max_blocks = (long long)ctx->num_sms * 8;  // 8 resident blocks of 256 threads per SM
   if (blocks > max_blocks) blocks = max_blocks;
   if (blocks < 1) blocks = 1;
-  kv_commit_kernel<<<(unsigned)blocks, kThreads, 0, static_cast<cudaStream_t>(stream)>>>(p);
+  DLM_CUDA_TRY(dlm_launch(kv_commit_kernel, dim3((unsigned)blocks), dim3(kThreads), 0, static_cast<cudaStream_t>(stream), p));
   return dlm_launch_ok(ctx, 1);
 }

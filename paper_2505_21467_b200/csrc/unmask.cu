@@ -232,6 +232,8 @@ template <int U>
 __global__ void __launch_bounds__(kThreads)
 vocab_reduce_kernel(const float* __restrict__ logits, int vocab, int chunk_len, int n_chunks, Triple* partial,
                     unsigned int* tickets, const SelectArgs sel) {
+  dlm_grid_dependency_wait();
+  dlm_trigger_dependents();
   const int row = blockIdx.y;
   if (sel.masked[row]) reduce_chunk<U>(logits, vocab, chunk_len, n_chunks, partial, row);
   if (tickets == nullptr) return;
@@ -253,6 +255,8 @@ vocab_reduce_kernel(const float* __restrict__ logits, int vocab, int chunk_len, 
 
 __global__ void __launch_bounds__(kThreads)
 unmask_select_kernel(const Triple* partial, int n_chunks, const SelectArgs sel) {
+  dlm_grid_dependency_wait();
+  dlm_trigger_dependents();
   select_batch(partial, n_chunks, blockIdx.x, sel);
 }
 
@@ -274,10 +278,12 @@ int launch_unmask(const float* logits, int batch, int block_len, int vocab, uint
   a.block_len = block_len; a.k = k; a.masked = masked; a.tokens = tokens; a.tok = tok; a.conf = conf;
   a.sel_idx = sel_idx; a.n_sel = n_sel;
   const dim3 grid(n_chunks, batch * block_len);
-  if (U == 4) vocab_reduce_kernel<4><<<grid, kThreads, 0, s>>>(logits, vocab, chunk_len, n_chunks, partial, tickets, a);
-  else vocab_reduce_kernel<8><<<grid, kThreads, 0, s>>>(logits, vocab, chunk_len, n_chunks, partial, tickets, a);
+  cudaError_t e;
+  if (U == 4) e = dlm_launch(vocab_reduce_kernel<4>, grid, dim3(kThreads), 0, s, logits, vocab, chunk_len, n_chunks, partial, tickets, a);
+  else e = dlm_launch(vocab_reduce_kernel<8>, grid, dim3(kThreads), 0, s, logits, vocab, chunk_len, n_chunks, partial, tickets, a);
+  if (e != cudaSuccess) return -1;
   if (tickets != nullptr) return 1;
-  unmask_select_kernel<<<batch, kThreads, 0, s>>>(partial, n_chunks, a);
+  if (dlm_launch(unmask_select_kernel, dim3(batch), dim3(kThreads), 0, s, partial, n_chunks, a) != cudaSuccess) return -1;
   return 2;
 }
 
@@ -304,6 +310,7 @@ extern "C" int dlm_unmask_select(dlm_ctx* ctx, const float* logits, int batch, i
   unsigned int* tickets = batch <= kDlmUnmaskTickets ? ctx->words->unmask_tickets : nullptr;
   const int n = launch_unmask(logits, batch, block_len, vocab, masked, tokens, k, tok, conf, sel_idx, n_sel,
                               static_cast<Triple*>(workspace), tickets, ctx->num_sms, static_cast<cudaStream_t>(stream));
+  if (n < 0) return DLM_ERR_CUDA;
   return dlm_launch_ok(ctx, n);
 }
 // ---------------------------------------------------------------------------------------
@@ -341,7 +348,8 @@ extern "C" int dlm_unmask_select_static(const float* logits, int batch, int bloc
       return DLM_ERR_CUDA;
     g_static_partial_addr[device] = addr;
   }
-  launch_unmask(logits, batch, block_len, vocab, masked, tokens, k, tok, conf, sel_idx, n_sel,
-                g_static_partial_addr[device], nullptr, 0, static_cast<cudaStream_t>(stream));
+  if (launch_unmask(logits, batch, block_len, vocab, masked, tokens, k, tok, conf, sel_idx, n_sel,
+                    g_static_partial_addr[device], nullptr, 0, static_cast<cudaStream_t>(stream)) < 0)
+    return DLM_ERR_CUDA;
   return cudaGetLastError() == cudaSuccess ? DLM_OK : DLM_ERR_CUDA;
 }
