@@ -96,6 +96,17 @@ def test_scores_that_keep_outgrowing_the_running_maximum(dev, oracle, scale):
         assert_attn_close(out, lse, ref[0], 0)
 
 
+def test_many_batch_elements_with_random_lengths(dev, oracle):
+    """600 sequences (the limit is 1024), each with its own cache length and window length, some empty."""
+    rng = np.random.default_rng(3)
+    B, Lcap, q_cap = 600, 70, 8
+    cache_len = rng.integers(0, Lcap + 1, B).tolist()
+    q_len = rng.integers(0, q_cap + 1, B).tolist()
+    out, lse, _ = _case(dev, oracle, 1, B, 2, 1, 64, Lcap, q_cap, cache_len, q_len, seed=606)
+    for b, n in enumerate(q_len):
+        assert torch.all(out[:, b, :, n:] == 0)
+
+
 def test_layer_range_and_explicit_scale(dev, oracle):
     _case(dev, oracle, 5, 1, 4, 2, 128, 300, 32, [290], seed=9, layer_begin=2, nl=2, scale=0.05)
 
