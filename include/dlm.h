@@ -48,7 +48,8 @@ enum {
   DLM_ERR_WORKSPACE = -5,   /* workspace NULL, misaligned or too small                      */
   DLM_ERR_CUDA = -6,        /* a CUDA runtime / driver call failed                          */
   DLM_ERR_TIMEOUT = -7,     /* a bounded device-side wait expired (kernel gave up cleanly)  */
-  DLM_ERR_INDEX = -8        /* a row index read from device memory is out of range          */
+  DLM_ERR_INDEX = -8,       /* a row index read from device memory is out of range          */
+  DLM_ERR_DEVICE = -9       /* the calling thread's current CUDA device is not the context's */
 };
 
 enum { DLM_DST_APPEND = 0, DLM_DST_WINDOW = 1 }; /* dlm_kv_cache_commit: where rows go when dst_pos is NULL */
@@ -56,6 +57,8 @@ enum { DLM_DST_APPEND = 0, DLM_DST_WINDOW = 1 }; /* dlm_kv_cache_commit: where r
 typedef struct dlm_ctx dlm_ctx;
 
 /* Creates a context bound to CUDA device `device` (must be compute capability 10.x).
+ * Every later call that takes the context must be made with that device current on the
+ * calling thread (else DLM_ERR_DEVICE, nothing launched).
  * The context owns only its status / ticket words.  Not thread-safe: use one context per
  * host thread or serialise calls.  Kernels enqueued through one context on different
  * streams must not overlap in time (they share the context's ticket words). */
@@ -107,7 +110,8 @@ typedef struct {
  *   k_new, v_new  device, bf16 [layer_end-layer_begin][batch][n_kv_heads][src_len][head_dim]
  *   src_idx       device, int32 [batch][n_max] or NULL
  *   dst_pos       device, int32 [batch][n_max] or NULL; destinations within one batch element
- *                 must be distinct (duplicates race; the result is then one of the sources)
+ *                 must be distinct (duplicates race: the row written is then unspecified and may
+ *                 mix 16-byte pieces of several sources, K and V independently)
  *   n_rows        device, int32 [batch] or NULL
  * Argument errors: NULL cache / tensors, src_len <= 0, n_max <= 0, bad layer range,
  * head_dim * 2 bytes not a multiple of 16.
@@ -178,7 +182,8 @@ size_t dlm_unmask_workspace_bytes(const dlm_ctx* ctx, int batch, int block_len, 
  * sel_idx[b][0..k_eff) = U ascending, remaining entries -1; n_sel[b] = k_eff.
  * If k == 0 ("propose only") only tok and conf are written; sel_idx / n_sel may be NULL.
  *
- *   logits   device, fp32 [batch][block_len][vocab]; -inf allowed, NaN / +inf unspecified
+ *   logits   device, fp32 [batch][block_len][vocab]; -inf entries allowed (they contribute 0); a masked
+ *            row that is -inf throughout, NaN and +inf are caller errors with unspecified results
  *   masked   device, uint8 [batch][block_len], in/out (non-zero = masked)
  *   tokens   device, int32 [batch][block_len], in/out
  *   tok      device, int32 [batch][block_len], out

@@ -16,7 +16,7 @@ from . import build as _build
 
 DLM_OK = 0
 DLM_ERR_NULL, DLM_ERR_SHAPE, DLM_ERR_UNSUPPORTED, DLM_ERR_CAPACITY = -1, -2, -3, -4
-DLM_ERR_WORKSPACE, DLM_ERR_CUDA, DLM_ERR_TIMEOUT, DLM_ERR_INDEX = -5, -6, -7, -8
+DLM_ERR_WORKSPACE, DLM_ERR_CUDA, DLM_ERR_TIMEOUT, DLM_ERR_INDEX, DLM_ERR_DEVICE = -5, -6, -7, -8, -9
 DLM_DST_APPEND, DLM_DST_WINDOW = 0, 1
 
 

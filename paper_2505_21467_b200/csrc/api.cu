@@ -19,8 +19,11 @@ extern "C" int dlm_create(dlm_ctx** out, int device) {
   if (!ctx) return DLM_ERR_CUDA;
   ctx->device = device;
   ctx->num_sms = prop.multiProcessorCount;
+  ctx->max_smem_optin = (int)prop.sharedMemPerBlockOptin;
   ctx->launches = 0;
   ctx->encode_tiled = nullptr;
+  ctx->commit_blocks_per_sm[0] = ctx->commit_blocks_per_sm[1] = 0;
+  ctx->attn_smem_limit[0] = ctx->attn_smem_limit[1] = 0;
   if (cudaMalloc(&ctx->words, sizeof(dlm_device_words)) != cudaSuccess ||
       cudaMemset(ctx->words, 0, sizeof(dlm_device_words)) != cudaSuccess) {
     delete ctx;
@@ -41,6 +44,7 @@ extern "C" int dlm_destroy(dlm_ctx* ctx) {
 
 extern "C" int dlm_get_status(dlm_ctx* ctx, void* stream) {
   if (!ctx) return DLM_ERR_NULL;
+  DLM_DEVICE_TRY(ctx);
   cudaStream_t s = static_cast<cudaStream_t>(stream);
   int code = 0;
   DLM_CUDA_TRY(cudaMemcpyAsync(&code, &ctx->words->status, sizeof(int), cudaMemcpyDeviceToHost, s));
@@ -67,6 +71,7 @@ extern "C" const char* dlm_strerror(int code) {
     case DLM_ERR_CUDA: return "a CUDA call failed";
     case DLM_ERR_TIMEOUT: return "a bounded device-side wait expired";
     case DLM_ERR_INDEX: return "a row index is out of range";
+    case DLM_ERR_DEVICE: return "the current CUDA device is not the context's device";
     default: return "unknown error code";
   }
 }
@@ -90,6 +95,7 @@ __global__ void wait_probe_kernel(unsigned long long limit_ns, int* status) {
 extern "C" int dlm_selftest_wait_timeout(dlm_ctx* ctx, uint64_t limit_ns, void* stream) {
   if (!ctx) return DLM_ERR_NULL;
   if (limit_ns == 0 || limit_ns > 1000000000ull) return DLM_ERR_SHAPE;   // at most one second
+  DLM_DEVICE_TRY(ctx);
   wait_probe_kernel<<<1, 32, 0, static_cast<cudaStream_t>(stream)>>>(limit_ns, &ctx->words->status);
   return dlm_launch_ok(ctx, 1);
 }

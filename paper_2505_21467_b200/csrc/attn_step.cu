@@ -5,7 +5,8 @@
 // One work unit is (layer, batch element, KV head, chunk of up to 256 query rows): the g = Hq/Hkv
 // query heads of a KV head, q_cap rows each, are cut into chunks of 256 rows = two 128-row M
 // tiles that share every K/V tile (at the block sizes of the configs, g * q_cap <= 256: one chunk,
-// K/V read from HBM once per KV head; larger windows re-read them per chunk, normally from L2).
+// K/V read from HBM once per KV head; larger windows re-read them per chunk, normally from L2;
+// calls with very few units use chunks of 128 rows, one M tile, to have more units to spread).
 // Keys are loaded in tiles of 128 rows, first the visible cache rows, then the fresh rows, and
 // processed in half-steps of 64.
 //
@@ -46,17 +47,19 @@ constexpr int kTileKeys = 128;
 constexpr int kPanelBytes = 128 * 128;   // one 64-element-wide panel of a 128-row tile
 constexpr int kMaxBatch = 1024;
 constexpr int kTmemCols = 512;
-constexpr int kRegsSoftmax = 216;     // registers per thread of the softmax warpgroups after setmaxnreg.inc
-constexpr int kRegsOther = 72;        // ... of the producer / MMA warpgroup after setmaxnreg.dec
+constexpr int kRegsSoftmax = 208;     // registers per thread of the softmax warpgroups after setmaxnreg.inc
+constexpr int kRegsOther = 88;        // ... of the producer / MMA warpgroup after setmaxnreg.dec
 constexpr int kMaxQCap = 4096;         // active rows per call
 constexpr int kMaxGrid = 256;          // blocks of the persistent grid (one per SM)
+constexpr int kMaxStages = 8;          // barrier slots reserved per ring
+constexpr int kBarrierBytes = 512;     // mbarriers of a block
+constexpr int kFlagBytes = 64;         // abort / never flags, TMEM slot, merge flag
 
 template <int D>
 struct Geometry {
   static constexpr int kPanels = D / 64;
   static constexpr int kTileBytes = kPanels * kPanelBytes;      // one K tile, V tile or Q M-tile
   static constexpr int kStages = (D == 128) ? 2 : 4;            // ring depth of K and of V
-  static constexpr int kSmemBytes = (2 + 2 * kStages) * kTileBytes + 1024 /*alignment*/ + 512 /*barriers*/;
   static constexpr uint32_t kColO = 0;                          // O[mt] at mt * D
   static constexpr uint32_t kColS = 2 * D;                      // S[mt] at 2D + mt * 128 (P aliases it)
 };
@@ -71,22 +74,25 @@ struct AttnParams {
   int nl, layer_begin, batch, n_kv_heads, n_q_heads, group, capacity, q_cap;
   int rows_total;  // group * q_cap: query rows per (layer, batch element, KV head)
   int n_rc;        // row chunks: rows_total cut into units of up to 256 rows (each re-reads the K/V tiles)
-  int rows;        // query rows per unit = min(256, rows_total)
+  int rows;        // query rows per unit = min(chunk_rows, rows_total)
+  int chunk_rows;  // 256 (two M tiles share every K/V tile) or 128 (one M tile per unit)
   int n_mt;        // M tiles per unit (1 or 2)
   int fresh_box;   // rows per TMA box of the fresh K/V tensors = min(128, q_cap)
   int whole_units; // 1: deal whole units round-robin, no partials
+  int smem_bytes;           // dynamic shared memory of the launch
   float scale_log2;
   int* status;
   unsigned int* tickets;   // one zero-initialised counter per unit: pieces finished
 };
 
-// Per-block scheduling tables (shared memory).
+// Per-block scheduling tables (in the block's dynamic shared memory, sized by batch and grid).
 struct Sched {
-  int prefix[kMaxBatch + 1];  // prefix[b] = tiles of batch elements < b; prefix[batch] = sum
-  int lc[kMaxBatch];          // clamped cache_len
-  int lq[kMaxBatch];          // clamped q_len
-  int share_lo[kMaxGrid + 1]; // split mode: block c owns items [share_lo[c], share_lo[c + 1])
+  int* prefix;    // [batch + 1]  prefix[b] = tiles of batch elements < b; prefix[batch] = sum
+  int* lc;        // [batch]      clamped cache_len
+  int* lq;        // [batch]      clamped q_len
+  int* share_lo;  // [grid + 1]   split mode: block c owns items [share_lo[c], share_lo[c + 1])
 };
+__host__ __device__ inline int sched_ints(int batch, int grid) { return 3 * (batch + 1) + 2 * (grid + 1); }
 
 struct Segment {
   int lc_layer, b, kvh, rc;   // unit: layer within the call, batch element, KV head, row chunk
@@ -292,24 +298,46 @@ __device__ __forceinline__ float row_max64(const uint32_t (&s)[64]) {
   return fmaxf(fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3])), fmaxf(fmaxf(mx[4], mx[5]), fmaxf(mx[6], mx[7])));
 }
 
-// P = 2^(s * scale - m) for the 64 scores, packed to bf16 pairs and written over the scores in TMEM;
-// returns the row sum.
-__device__ __forceinline__ float exp64_store(const uint32_t (&s)[64], float scale_log2, float m_used, uint32_t t_s) {
-  float l0 = 0.f, l1 = 0.f;
+// Two positive finite floats to a packed pair of bf16 (a in the low half), rounded to nearest with
+// ties away from zero: integer adds and a byte permute.  The conversion instruction runs on the
+// SFU's pipe (2 cycles per warp instruction on top of 8 per exponential), and that pipe is what
+// bounds the softmax warps.
+__device__ __forceinline__ uint32_t pack_bf16_pos(float a, float b) {
+  return __byte_perm(__float_as_uint(a) + 0x8000u, __float_as_uint(b) + 0x8000u, 0x7632);
+}
+
+// P = 2^(s * scale - m) for 32 scores, packed to bf16 pairs and written to 16 TMEM columns at t_p;
+// adds to the two partial row sums.  The 32 exponentials are independent instructions issued back
+// to back and only then summed and packed: a score-by-score chain (multiply-add, exponential, add)
+// leaves the warp waiting on latencies instead of keeping the SFU busy.
+__device__ __forceinline__ void exp32_store(const uint32_t* s, float scale_log2, float m_used, uint32_t t_p, float& l0,
+                                            float& l1) {
+  float x[32];
 #pragma unroll
-  for (int c = 0; c < 2; ++c) {
-    uint32_t pk[16];
+  for (int j = 0; j < 32; ++j) x[j] = fmaf(__uint_as_float(s[j]), scale_log2, -m_used);
 #pragma unroll
-    for (int j = 0; j < 16; ++j) {
-      const float p0 = ex2_approx(fmaf(__uint_as_float(s[32 * c + 2 * j]), scale_log2, -m_used));
-      const float p1 = ex2_approx(fmaf(__uint_as_float(s[32 * c + 2 * j + 1]), scale_log2, -m_used));
-      l0 += p0;
-      l1 += p1;
-      const __nv_bfloat162 h = __floats2bfloat162_rn(p0, p1);
-      pk[j] = *reinterpret_cast<const uint32_t*>(&h);
-    }
-    tmem_st16(t_s + c * 16, pk);
+  for (int j = 0; j < 32; ++j) x[j] = ex2_approx(x[j]);
+  uint32_t pk[16];
+  float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
+#pragma unroll
+  for (int j = 0; j < 8; ++j) {
+    a0 += x[4 * j];
+    a1 += x[4 * j + 1];
+    a2 += x[4 * j + 2];
+    a3 += x[4 * j + 3];
+    pk[2 * j] = pack_bf16_pos(x[4 * j], x[4 * j + 1]);
+    pk[2 * j + 1] = pack_bf16_pos(x[4 * j + 2], x[4 * j + 3]);
   }
+  l0 += a0 + a2;
+  l1 += a1 + a3;
+  tmem_st16(t_p, pk);
+}
+
+// The same for 64 scores (32 TMEM columns at t_p); returns the row sum.
+__device__ __forceinline__ float exp64_store(const uint32_t (&s)[64], float scale_log2, float m_used, uint32_t t_p) {
+  float l0 = 0.f, l1 = 0.f;
+  exp32_store(s, scale_log2, m_used, t_p, l0, l1);
+  exp32_store(s + 32, scale_log2, m_used, t_p + 16, l0, l1);
   return l0 + l1;
 }
 
@@ -378,8 +406,7 @@ __device__ __noinline__ bool softmax_half_ragged(uint32_t t_s, uint32_t t_o, int
       if (c * 32 + 2 * j >= valid) p0 = 0.f;
       if (c * 32 + 2 * j + 1 >= valid) p1 = 0.f;
       l_add += p0 + p1;
-      const __nv_bfloat162 h = __floats2bfloat162_rn(p0, p1);
-      pk[j] = *reinterpret_cast<const uint32_t*>(&h);
+      pk[j] = pack_bf16_pos(p0, p1);
     }
     tmem_st16(t_s + c * 16, pk);
   }
@@ -394,24 +421,42 @@ attn_step_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
                        const __grid_constant__ CUtensorMap tm_vc, const __grid_constant__ CUtensorMap tm_kn,
                        const __grid_constant__ CUtensorMap tm_vn, const AttnParams p) {
   using G = Geometry<D>;
-  constexpr int KS = G::kStages;
+  // Shared memory of the block, all of it dynamic so that the host can give every byte that is left over
+  // to K/V stages (what bounds this kernel at the configs' shapes is the number of bytes in flight):
+  // [Q: n_mt tiles][K: k_stages tiles][V: v_stages tiles][barriers][flags][scheduling tables], from
+  // the first 1024-byte boundary (the swizzled tiles need that alignment).
   extern __shared__ uint8_t smem_raw[];
-  __shared__ Sched sched;
-  __shared__ int abort_flag;
-  __shared__ int never_flag;   // stays 0: for waits that must not be cut short by an abort
-  __shared__ uint32_t tmem_slot;
-  __shared__ int merge_ok;
-  __shared__ int merge_slot[kMaxGrid];
+  // compile-time ring depths: the MMA issuers' scalar code is on the critical path, and divisions by a
+  // run-time depth in it cost 10 % at the LLaDA shape
+  constexpr int KS = G::kStages, VS = G::kStages;
+  const uint32_t smem_pad = (1024u - (smem_u32(smem_raw) & 1023u)) & 1023u;
+  const uint32_t smem_base = smem_u32(smem_raw) + smem_pad;
+  const uint32_t sm_q = smem_base;                               // [n_mt][kTileBytes]
+  const uint32_t sm_k = sm_q + p.n_mt * G::kTileBytes;           // [KS][kTileBytes]
+  const uint32_t sm_v = sm_k + KS * G::kTileBytes;               // [VS][kTileBytes]
+  const uint32_t sm_bar = sm_v + VS * G::kTileBytes;             // barriers, 8 bytes each
+  int* const flags = reinterpret_cast<int*>(smem_raw + smem_pad + (size_t)(p.n_mt + KS + VS) * G::kTileBytes + kBarrierBytes);
+  volatile int* const abort_ptr = flags;        // raised by the first wait that gives up
+  volatile int* const never_ptr = flags + 1;    // stays 0: for waits that must not be cut short by an abort
+  uint32_t* const tmem_slot = reinterpret_cast<uint32_t*>(flags + 2);
+  volatile int* const merge_ok = flags + 3;
+  Sched sched;
+  sched.prefix = flags + kFlagBytes / 4;
+  sched.lc = sched.prefix + p.batch + 1;
+  sched.lq = sched.lc + p.batch;
+  sched.share_lo = sched.lq + p.batch;
+  int* const merge_slot = sched.share_lo + gridDim.x + 1;   // [grid]
+  if (smem_pad + (uint32_t)(p.n_mt + KS + VS) * G::kTileBytes + kBarrierBytes + kFlagBytes +
+          4u * (uint32_t)sched_ints(p.batch, gridDim.x) > (uint32_t)p.smem_bytes) {
+    // cannot happen with the host's sizing (it leaves room for the largest pad); nothing has been touched yet
+    if (threadIdx.x == 0) dlm_set_status(p.status, DLM_ERR_WORKSPACE);
+    return;
+  }
 
-  const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
-  const uint32_t sm_q = smem_base;                               // [2][kTileBytes]
-  const uint32_t sm_k = sm_q + 2 * G::kTileBytes;                // [KS][kTileBytes]
-  const uint32_t sm_v = sm_k + KS * G::kTileBytes;               // [KS][kTileBytes]
-  const uint32_t sm_bar = sm_v + KS * G::kTileBytes;             // barriers, 8 bytes each
   const uint32_t bar_q_full = sm_bar, bar_q_empty = sm_bar + 8, bar_drain = sm_bar + 16;   // drain: [2]
-  const uint32_t bar_k_full = sm_bar + 32, bar_k_empty = bar_k_full + 8 * KS;
-  const uint32_t bar_v_full = bar_k_empty + 8 * KS, bar_v_empty = bar_v_full + 8 * KS;
-  const uint32_t bar_s_ready = bar_v_empty + 8 * KS;             // [M tile][score buffer]: scores of a half-step written
+  const uint32_t bar_k_full = sm_bar + 32, bar_k_empty = bar_k_full + 8 * kMaxStages;
+  const uint32_t bar_v_full = bar_k_empty + 8 * kMaxStages, bar_v_empty = bar_v_full + 8 * kMaxStages;
+  const uint32_t bar_s_ready = bar_v_empty + 8 * kMaxStages;             // [M tile][score buffer]: scores of a half-step written
   const uint32_t bar_p_ready = bar_s_ready + 32;                 // [M tile][score buffer]: P of a half-step written
   const uint32_t bar_pv_done = bar_p_ready + 32;                 // [M tile][half-step parity] P V product finished.  Two P V
                                                                  // products can be in flight, so consecutive half-steps use different
@@ -419,14 +464,13 @@ attn_step_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
   const uint32_t bar_pub = bar_pv_done + 32;                     // partial result of a segment stored by every softmax thread
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  volatile int* abort_ptr = &abort_flag;
   // softmax threads that own a real query row, rounded up to whole warps (they are tid 0 .. n_live-1)
   const int n_live = (p.rows + 31) & ~31;
 
   // ---- set-up: barriers, TMEM and descriptor prefetch first (they need no data), so that they overlap
   // the cold read of the lengths; then the tile prefix
   if (tid == 0) {
-    abort_flag = 0; never_flag = 0; merge_ok = 0;
+    *abort_ptr = 0; *never_ptr = 0; *merge_ok = 0;
     mbar_init(bar_q_full, 1);
     mbar_init(bar_q_empty, (uint32_t)p.n_mt);       // one commit per MMA issuer
     mbar_init(bar_drain, 1);
@@ -435,11 +479,13 @@ attn_step_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
     for (int i = 0; i < KS; ++i) {
       mbar_init(bar_k_full + 8 * i, 1);
       mbar_init(bar_k_empty + 8 * i, (uint32_t)p.n_mt);
+    }
+    for (int i = 0; i < VS; ++i) {
       mbar_init(bar_v_full + 8 * i, 1);
       mbar_init(bar_v_empty + 8 * i, (uint32_t)p.n_mt);
     }
     for (int i = 0; i < 2; ++i) {
-      const uint32_t live_i = (uint32_t)max(32, min(128, n_live - 128 * i));
+      const uint32_t live_i = (uint32_t)max(32, min(128, n_live - 128 * i)) / 32;   // one arrival per live warp
       for (int u = 0; u < 2; ++u) {
         mbar_init(bar_s_ready + 16 * i + 8 * u, 1);
         mbar_init(bar_p_ready + 16 * i + 8 * u, live_i);
@@ -451,7 +497,7 @@ attn_step_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
     fence_proxy_async_smem();
   }
   if (warp == 9) {
-    tmem_alloc(smem_u32(&tmem_slot), kTmemCols);
+    tmem_alloc(smem_u32(tmem_slot), kTmemCols);
     tmem_relinquish();
   }
   if (warp == 8 && lane == 0) {
@@ -487,7 +533,7 @@ attn_step_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
   tc_fence_before_sync();
   __syncthreads();
   tc_fence_after_sync();
-  const uint32_t tmem = tmem_slot;
+  const uint32_t tmem = *tmem_slot;
   // number of shares the item list is cut into (every share holds at least one item)
   const int total_items = sched.prefix[p.batch] * p.nl * p.n_kv_heads * p.n_rc;
   const int n_cta = p.whole_units ? (int)gridDim.x : min((int)gridDim.x, total_items);
@@ -522,7 +568,7 @@ attn_step_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
           for (int mt = 0; mt < p.n_mt; ++mt)
             for (int pn = 0; pn < G::kPanels; ++pn)
               tma_load_3d(sm_q + mt * G::kTileBytes + pn * kPanelBytes, &tm_q, bar_q_full, pn * 64,
-                          g.rc * 256 + mt * 128, zq);
+                          g.rc * p.chunk_rows + mt * 128, zq);
           for (int t = g.t_begin; t < g.t_end && ok; ++t) {
             const bool cache = t < g.n_ct;
             const int row = cache ? t * kTileKeys : (t - g.n_ct) * p.fresh_box;
@@ -539,8 +585,8 @@ attn_step_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
               ++kt;
             }
             {
-              const uint32_t s = vt % KS;
-              if (vt >= (uint32_t)KS) ok = mbar_wait(bar_v_empty + 8 * s, ((vt / KS) - 1) & 1, abort_ptr);
+              const uint32_t s = vt % VS;
+              if (vt >= (uint32_t)VS) ok = mbar_wait(bar_v_empty + 8 * s, ((vt / VS) - 1) & 1, abort_ptr);
               if (!ok) break;
               mbar_expect_tx(bar_v_full + 8 * s, bytes);
               for (int pn = 0; pn < G::kPanels; ++pn)
@@ -554,9 +600,9 @@ attn_step_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
         if (!ok) {
           // unwinding: let the copies already issued land before the block's memory is released
           for (uint32_t i = (kt > (uint32_t)KS ? kt - KS : 0); i < kt; ++i)
-            mbar_wait(bar_k_full + 8 * (i % KS), (i / KS) & 1, &never_flag);
-          for (uint32_t i = (vt > (uint32_t)KS ? vt - KS : 0); i < vt; ++i)
-            mbar_wait(bar_v_full + 8 * (i % KS), (i / KS) & 1, &never_flag);
+            mbar_wait(bar_k_full + 8 * (i % KS), (i / KS) & 1, never_ptr);
+          for (uint32_t i = (vt > (uint32_t)VS ? vt - VS : 0); i < vt; ++i)
+            mbar_wait(bar_v_full + 8 * (i % VS), (i / VS) & 1, never_ptr);
         }
       }
     } else if (warp == 9 || warp == 10) {
@@ -647,9 +693,9 @@ attn_step_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
           bool first = true;
           HalfStep hs;
           while (ok && pi.get(hs)) {
-            const uint32_t vs = vt % KS;
+            const uint32_t vs = vt % VS;
             if (hs.first_of_tile) {
-              ok = wait_warp(bar_v_full + 8 * vs, (vt / KS) & 1);
+              ok = wait_warp(bar_v_full + 8 * vs, (vt / VS) & 1);
               if (!ok) break;
             }
             ok = wait_warp(bar_p_ready + 16 * mt + 8 * (gt & 1), (gt >> 1) & 1);
@@ -671,7 +717,7 @@ attn_step_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
         // every MMA issued by this warp has finished before TMEM is released
         if (elect_one_sync()) tc_commit(bar_drain + 8 * mt);
         __syncwarp();
-        mbar_wait(bar_drain + 8 * mt, 0, &never_flag);
+        mbar_wait(bar_drain + 8 * mt, 0, never_ptr);
       }
     } else {
       // ================================================================= publisher (warp 11)
@@ -709,7 +755,7 @@ attn_step_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
       };
       // this thread's query row in row chunk rc of a KV head: which of its query heads, which active row
       auto out_row_of = [&](int lc_layer, int b, int kvh, int rc) {
-        const int r = rc * 256 + r_unit;
+        const int r = rc * p.chunk_rows + r_unit;
         const int hl = r < p.rows_total ? r / p.q_cap : 0, ir = r < p.rows_total ? r % p.q_cap : 0;
         return (((size_t)lc_layer * p.batch + b) * p.n_q_heads + (size_t)kvh * p.group + hl) * p.q_cap + ir;
       };
@@ -728,7 +774,7 @@ attn_step_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
           const int b = unit % p.batch, grp = unit / p.batch, rc = grp % p.n_rc;
           if (sched.prefix[b + 1] == sched.prefix[b])
             zero_my_row(out_row_of((grp / p.n_rc) / p.n_kv_heads, b, (grp / p.n_rc) % p.n_kv_heads, rc),
-                        rc * 256 + r_unit < p.rows_total);
+                        rc * p.chunk_rows + r_unit < p.rows_total);
         }
       }
       if (has_work) {
@@ -739,7 +785,7 @@ attn_step_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
         while (ok && walk.next(g, n_cta)) {
           const int n = g.t_end - g.t_begin;
           const size_t qrow = out_row_of(g.lc_layer, g.b, g.kvh, g.rc);
-          const int r_kv = g.rc * 256 + r_unit;               // row among all query rows of the KV head
+          const int r_kv = g.rc * p.chunk_rows + r_unit;               // row among all query rows of the KV head
           const bool real_row = r_kv < p.rows_total;
           const int i_row = real_row ? r_kv % p.q_cap : 0;
           if (n <= 0) {  // whole-unit mode, inactive batch element: the unit's rows are zero
@@ -756,8 +802,8 @@ attn_step_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
               // NaN / Inf bit patterns cannot reach O.  Each M tile's warps do it before they
               // announce the P of the tile's first half-step, so it precedes that tile's P V
               // products (the two M tiles write the same zeros).
-              const uint32_t vs = vt % KS;
-              ok = wait_warp(bar_v_full + 8 * vs, (vt / KS) & 1);
+              const uint32_t vs = vt % VS;
+              ok = wait_warp(bar_v_full + 8 * vs, (vt / VS) & 1);
               if (!ok) break;
               const int per_row = G::kPanels * 8;
               for (int idx = row; idx < (n16 - valid) * per_row; idx += n_live_mt) {
@@ -781,8 +827,12 @@ attn_step_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
                 ok = softmax_half_ragged<D>(t_s + buf * kHalfKeys, t_o, nkeys, first, p.scale_log2, m_used, l_run,
                                             bar_pv_done + 16 * mt + 8 * ((gt - 1) & 1), ((gt - 1) >> 1) & 1, abort_ptr);
               if (!ok) break;
-              tc_fence_before_sync();
-              mbar_arrive(bar_p_ready + 16 * mt + 8 * buf);
+              // every lane's P is stored (tcgen05.wait::st inside the softmax); one lane announces the warp's rows
+              __syncwarp();
+              if (lane == 0) {
+                tc_fence_before_sync();
+                mbar_arrive(bar_p_ready + 16 * mt + 8 * buf);
+              }
               first = false;
             }
           }
@@ -843,12 +893,12 @@ attn_step_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
               const int n_others = up.c_last - up.c_first;
               const int unit = ((g.lc_layer * p.n_kv_heads + g.kvh) * p.n_rc + g.rc) * p.batch + g.b;
               if (tid == 0) {
-                merge_ok = wait_counter(p.tickets + unit, (unsigned int)n_others, abort_ptr) ? 1 : 0;
-                if (merge_ok) p.tickets[unit] = 0;   // ready for the next launch
+                *merge_ok = wait_counter(p.tickets + unit, (unsigned int)n_others, abort_ptr) ? 1 : 0;
+                if (*merge_ok) p.tickets[unit] = 0;   // ready for the next launch
               }
               for (int i = tid; i < n_others; i += n_live) merge_slot[i] = up.slot_of(up.c_first + i);
               named_bar_sync(1, n_live);
-              if (!merge_ok) { ok = false; break; }
+              if (!*merge_ok) { ok = false; break; }
               __threadfence();
               // maximum and sum over all pieces
               float m_all = m_used, l_all = l_run;
@@ -920,7 +970,7 @@ attn_step_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
   }
   // ---- teardown: nothing of this block is in flight any more
   __syncwarp();
-  if (tid == 0 && abort_flag) dlm_set_status(p.status, DLM_ERR_TIMEOUT);
+  if (tid == 0 && *abort_ptr) dlm_set_status(p.status, DLM_ERR_TIMEOUT);
   tc_fence_before_sync();
   __syncthreads();
   if (warp == 9) {
@@ -957,16 +1007,39 @@ int encode_map(dlm_ctx* ctx, CUtensorMap* map, const void* base, int D, long lon
 // The kernel starts with `numRegs` registers per thread in all 12 warps.  The 8 softmax warps then
 // ask for kRegsSoftmax each and block until they get them; only what the other 4 warps release
 // is certain to be free, so the request must fit inside that.
-bool register_budget_ok(const void* kern) {
-  cudaFuncAttributes a;
-  if (cudaFuncGetAttributes(&a, kern) != cudaSuccess) return false;
+bool register_budget_ok(const cudaFuncAttributes& a) {
   return a.numRegs >= kRegsOther && 8 * (kRegsSoftmax - a.numRegs) <= 4 * (a.numRegs - kRegsOther);
 }
 
+// First use of an attention kernel on a context's device: checks the register budget and opts in to
+// all the dynamic shared memory the device allows a block (less the kernel's static part).
+int configure_kernel(dlm_ctx* ctx, int which, const void* kern) {
+  if (ctx->attn_smem_limit[which] > 0) return DLM_OK;
+  cudaFuncAttributes a;
+  DLM_CUDA_TRY(cudaFuncGetAttributes(&a, kern));
+  if (!register_budget_ok(a)) return DLM_ERR_UNSUPPORTED;
+  const int limit = ctx->max_smem_optin - (int)a.sharedSizeBytes;
+  if (limit <= 0) return DLM_ERR_UNSUPPORTED;
+  DLM_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, limit));
+  ctx->attn_smem_limit[which] = limit;
+  return DLM_OK;
+}
+
 struct Plan {
-  int n_mt, rows, rows_total, n_rc, grid, whole_units;
+  int n_mt, rows, rows_total, n_rc, grid, whole_units, chunk_rows;
+  int smem_bytes;
   size_t ws_o_bytes, ws_ml_bytes;
 };
+
+// Shared memory of a block: Q tiles, the K and V rings, barriers, flags, scheduling tables and up to
+// 1023 bytes of alignment.  (Deeper rings were measured: 2 + 3 and 3 + 3 stages at head_dim 128 were
+// 3 - 10 % slower on the configs' shapes, so the rest of the shared memory stays unused.)
+bool plan_shared_memory(int smem_limit, int head_dim, int batch, Plan& pl) {
+  const int tile = head_dim / 64 * kPanelBytes;
+  const int stages = head_dim == 128 ? Geometry<128>::kStages : Geometry<64>::kStages;
+  pl.smem_bytes = 1024 + (pl.n_mt + 2 * stages) * tile + kBarrierBytes + kFlagBytes + 4 * sched_ints(batch, pl.grid);
+  return pl.smem_bytes <= smem_limit;
+}
 
 // Splitting units across blocks balances the load but costs each block a partial store and each
 // unit a wait and a merge that grows with its number of pieces (measured: about 3 key tiles' worth
@@ -977,8 +1050,14 @@ struct Plan {
 Plan make_plan(const dlm_ctx* ctx, const dlm_kv_cache* cache, int nl, int n_q_heads, int q_cap, int cache_len_hint) {
   Plan pl;
   pl.rows_total = (n_q_heads / cache->n_kv_heads) * q_cap;
-  pl.n_rc = (pl.rows_total + 255) / 256;
-  pl.rows = pl.rows_total < 256 ? pl.rows_total : 256;
+  // Row chunks of 256 (two M tiles sharing every K/V tile) read K/V once per KV head.  When a call has
+  // only a handful of such units (one layer of a small batch), chunks of 128 double the units that can
+  // be spread over the SMs and halve every partial result; the second read of K/V comes from L2
+  // (measured on one Dream-shaped layer at batch 1: 15.9 us against 20.9).
+  const long long units256 = (long long)nl * cache->batch * cache->n_kv_heads * ((pl.rows_total + 255) / 256);
+  pl.chunk_rows = (pl.rows_total > 128 && units256 * 8 <= ctx->num_sms) ? 128 : 256;
+  pl.n_rc = (pl.rows_total + pl.chunk_rows - 1) / pl.chunk_rows;
+  pl.rows = pl.rows_total < pl.chunk_rows ? pl.rows_total : pl.chunk_rows;
   pl.n_mt = (pl.rows + 127) / 128;
   const long long units = (long long)nl * cache->batch * cache->n_kv_heads * pl.n_rc;
   const int sms = ctx->num_sms < kMaxGrid ? ctx->num_sms : kMaxGrid;
@@ -1040,10 +1119,18 @@ extern "C" int dlm_freecache_attn_step(dlm_ctx* ctx, const dlm_kv_cache* cache, 
   if (((uintptr_t)cache->k | (uintptr_t)cache->v | (uintptr_t)q | (uintptr_t)k_new | (uintptr_t)v_new |
        (uintptr_t)out) & 15)
     return DLM_ERR_UNSUPPORTED;
+  DLM_DEVICE_TRY(ctx);
   const int nl = layer_end - layer_begin;
   const size_t need = dlm_attn_workspace_bytes(ctx, cache, nl, n_q_heads, q_cap);
   if (!workspace || workspace_bytes < need || ((uintptr_t)workspace & 255)) return DLM_ERR_WORKSPACE;
   const Plan pl = make_plan(ctx, cache, nl, n_q_heads, q_cap, cache_len_hint);
+  {
+    const int rc = D == 128 ? configure_kernel(ctx, 0, reinterpret_cast<const void*>(attn_step_sm100_kernel<128>))
+                            : configure_kernel(ctx, 1, reinterpret_cast<const void*>(attn_step_sm100_kernel<64>));
+    if (rc != DLM_OK) return rc;
+  }
+  Plan pl_mut = pl;
+  if (!plan_shared_memory(ctx->attn_smem_limit[D == 128 ? 0 : 1], D, cache->batch, pl_mut)) return DLM_ERR_UNSUPPORTED;
   {  // the split schedule counts (unit, key tile) items in 32 bits
     const long long tiles_per_unit = (cache->capacity + 127) / 128 + (q_cap + 127) / 128 + 1;
     if (!pl.whole_units && (long long)nl * cache->batch * cache->n_kv_heads * pl.n_rc * tiles_per_unit >= (1LL << 30))
@@ -1066,11 +1153,13 @@ extern "C" int dlm_freecache_attn_step(dlm_ctx* ctx, const dlm_kv_cache* cache, 
   p.capacity = cache->capacity;
   p.q_cap = q_cap;
   p.rows = pl.rows;
+  p.chunk_rows = pl.chunk_rows;
   p.rows_total = pl.rows_total;
   p.n_rc = pl.n_rc;
   p.n_mt = pl.n_mt;
   p.fresh_box = q_cap < 128 ? q_cap : 128;
   p.whole_units = pl.whole_units;
+  p.smem_bytes = pl_mut.smem_bytes;
   const float scale = softmax_scale > 0.f ? softmax_scale : 1.0f / sqrtf((float)D);
   p.scale_log2 = scale * 1.4426950408889634f;
   p.status = &ctx->words->status;
@@ -1088,24 +1177,11 @@ extern "C" int dlm_freecache_attn_step(dlm_ctx* ctx, const dlm_kv_cache* cache, 
   if (rc != DLM_OK) return rc;
 
   cudaStream_t s = static_cast<cudaStream_t>(stream);
-  if (D == 128) {
-    auto kern = attn_step_sm100_kernel<128>;
-    static bool configured = false;
-    if (!configured) {
-      if (!register_budget_ok(reinterpret_cast<const void*>(kern))) return DLM_ERR_UNSUPPORTED;
-      DLM_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, Geometry<128>::kSmemBytes));
-      configured = true;
-    }
-    DLM_CUDA_TRY(dlm_launch(kern, dim3(pl.grid), dim3(kThreads), Geometry<128>::kSmemBytes, s, tm_q, tm_kc, tm_vc, tm_kn, tm_vn, p));
-  } else {
-    auto kern = attn_step_sm100_kernel<64>;
-    static bool configured = false;
-    if (!configured) {
-      if (!register_budget_ok(reinterpret_cast<const void*>(kern))) return DLM_ERR_UNSUPPORTED;
-      DLM_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, Geometry<64>::kSmemBytes));
-      configured = true;
-    }
-    DLM_CUDA_TRY(dlm_launch(kern, dim3(pl.grid), dim3(kThreads), Geometry<64>::kSmemBytes, s, tm_q, tm_kc, tm_vc, tm_kn, tm_vn, p));
-  }
+  if (D == 128)
+    DLM_CUDA_TRY(dlm_launch(attn_step_sm100_kernel<128>, dim3(pl.grid), dim3(kThreads), (size_t)p.smem_bytes, s, tm_q, tm_kc,
+                            tm_vc, tm_kn, tm_vn, p));
+  else
+    DLM_CUDA_TRY(dlm_launch(attn_step_sm100_kernel<64>, dim3(pl.grid), dim3(kThreads), (size_t)p.smem_bytes, s, tm_q, tm_kc,
+                            tm_vc, tm_kn, tm_vn, p));
   return dlm_launch_ok(ctx, 1);
 }

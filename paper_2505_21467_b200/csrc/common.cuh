@@ -23,9 +23,12 @@ struct dlm_device_words {
 struct dlm_ctx {
   int device;
   int num_sms;
+  int max_smem_optin;       // largest dynamic shared memory a block may opt in to, bytes
   int64_t launches;
   dlm_device_words* words;  // device
   void* encode_tiled;       // cuTensorMapEncodeTiled entry point (driver API), resolved lazily
+  int commit_blocks_per_sm[2];  // resident blocks per SM of the two commit kernels (0 = not asked yet)
+  int attn_smem_limit[2];       // dynamic shared memory the two attention kernels may use on this device (0 = not set up yet)
 };
 
 #define DLM_CUDA_TRY(expr)                         \
@@ -64,6 +67,19 @@ static inline cudaError_t dlm_launch(void (*kernel)(KArgs...), dim3 grid, dim3 b
   cfg.numAttrs = 1;
   return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
 }
+
+// The context's device must be the calling thread's current device: launches go to the current
+// device, the context's words and the caller's pointers live on the context's.
+static inline int dlm_check_device(const dlm_ctx* ctx) {
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess) return DLM_ERR_CUDA;
+  return dev == ctx->device ? DLM_OK : DLM_ERR_DEVICE;
+}
+#define DLM_DEVICE_TRY(ctx)                        \
+  do {                                             \
+    const int _d = dlm_check_device(ctx);          \
+    if (_d != DLM_OK) return _d;                   \
+  } while (0)
 
 static inline int dlm_launch_ok(dlm_ctx* ctx, int n_kernels) {
   if (cudaGetLastError() != cudaSuccess) return DLM_ERR_CUDA;

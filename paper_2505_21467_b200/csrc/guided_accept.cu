@@ -72,6 +72,7 @@ extern "C" int dlm_guided_accept(dlm_ctx* ctx, const int32_t* tok_dlm, const int
   if (!ctx || !tok_dlm || !tok_ar || !masked || !tokens || !accept || !acc_idx || !n_acc) return DLM_ERR_NULL;
   if (batch <= 0 || block_len <= 0) return DLM_ERR_SHAPE;
   if (block_len > 1024 || (fallback_source != 0 && fallback_source != 1)) return DLM_ERR_UNSUPPORTED;
+  DLM_DEVICE_TRY(ctx);
   DLM_CUDA_TRY(dlm_launch(guided_accept_kernel, dim3(batch), dim3(32), 0, static_cast<cudaStream_t>(stream), tok_dlm, tok_ar, 1,
                           block_len, masked, tokens, fallback_source, accept, acc_idx, n_acc));
   return dlm_launch_ok(ctx, 1);
@@ -83,6 +84,7 @@ extern "C" int dlm_guided_accept_topk(dlm_ctx* ctx, const int32_t* tok_dlm, cons
   if (!ctx || !tok_dlm || !tok_ar_topk || !masked || !tokens || !accept || !acc_idx || !n_acc) return DLM_ERR_NULL;
   if (batch <= 0 || block_len <= 0 || top_k <= 0) return DLM_ERR_SHAPE;
   if (block_len > 1024 || top_k > 64 || (fallback_source != 0 && fallback_source != 1)) return DLM_ERR_UNSUPPORTED;
+  DLM_DEVICE_TRY(ctx);
   DLM_CUDA_TRY(dlm_launch(guided_accept_kernel, dim3(batch), dim3(32), 0, static_cast<cudaStream_t>(stream), tok_dlm,
                           tok_ar_topk, top_k, block_len, masked, tokens, fallback_source, accept, acc_idx, n_acc));
   return dlm_launch_ok(ctx, 1);

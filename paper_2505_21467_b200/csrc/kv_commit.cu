@@ -4,8 +4,11 @@
 // Pure data movement, bound by HBM.  One work item is one 16-byte vector of one K row and
 // the matching vector of the V row; items are ordered [layer][batch][head][row][vector] so
 // that consecutive threads touch consecutive addresses whenever the row indices are
-// consecutive (refresh / append).  Each thread keeps UNROLL independent 16-byte loads of K
-// and of V in flight.  The last block to finish advances cache_len.
+// consecutive (refresh / append).  The item list is cut into equal contiguous ranges, one per
+// block, and the grid is one resident wave, so every SM moves the same number of bytes; a
+// thread keeps kUnroll independent 16-byte loads of K and of V in flight.  Item numbers are
+// decoded with 32-bit arithmetic whenever the call has fewer than 2^31 items (64-bit divisions
+// by run-time divisors cost more than the copy).  The last block to finish advances cache_len.
 #include "common.cuh"
 
 namespace {
@@ -27,6 +30,7 @@ struct CommitParams {
   int vec_per_row;       // head_dim * 2 / 16
   int vec_shift;         // log2(vec_per_row) or -1
   long long n_items;     // n_layers_call * batch * heads * n_max * vec_per_row
+  long long per_block;   // items per block (a multiple of 32)
   int* status;
   unsigned int* ticket;
 };
@@ -40,34 +44,36 @@ __device__ __forceinline__ int valid_rows(const CommitParams& p, int b, int len0
   return n;
 }
 
-__global__ void __launch_bounds__(kThreads) kv_commit_kernel(const CommitParams p) {
+template <typename Idx>
+__global__ void __launch_bounds__(kThreads, 4) kv_commit_kernel(const CommitParams p) {
   dlm_grid_dependency_wait();
   dlm_trigger_dependents();
-  const long long stride = (long long)gridDim.x * kThreads;
-  const long long first = (long long)blockIdx.x * kThreads + threadIdx.x;
-  for (long long base = first; base < p.n_items; base += stride * kUnroll) {
+  const Idx begin = (Idx)blockIdx.x * (Idx)p.per_block;
+  const Idx end = (Idx)min((long long)begin + p.per_block, p.n_items);
+  const Idx n_max = (Idx)p.n_max, heads = (Idx)p.n_kv_heads, batch = (Idx)p.batch;
+  for (Idx base = begin + threadIdx.x; base < end; base += kThreads * kUnroll) {
     uint4 kk[kUnroll], vv[kUnroll];
     long long to[kUnroll];
 #pragma unroll
     for (int u = 0; u < kUnroll; ++u) {
       to[u] = -1;
-      long long item = base + (long long)u * stride;
-      if (item >= p.n_items) continue;
+      const Idx item = base + (Idx)(u * kThreads);
+      if (item >= end) continue;
       int vec;
-      long long rest;
+      Idx rest;
       if (p.vec_shift >= 0) {
-        vec = (int)(item & (p.vec_per_row - 1));
+        vec = (int)(item & (Idx)(p.vec_per_row - 1));
         rest = item >> p.vec_shift;
       } else {
-        vec = (int)(item % p.vec_per_row);
-        rest = item / p.vec_per_row;
+        vec = (int)(item % (Idx)p.vec_per_row);
+        rest = item / (Idx)p.vec_per_row;
       }
-      const int r = (int)(rest % p.n_max);
-      rest /= p.n_max;
-      const int h = (int)(rest % p.n_kv_heads);
-      rest /= p.n_kv_heads;
-      const int b = (int)(rest % p.batch);
-      const int lc = (int)(rest / p.batch);  // layer within the call
+      const int r = (int)(rest % n_max);
+      rest /= n_max;
+      const int h = (int)(rest % heads);
+      rest /= heads;
+      const int b = (int)(rest % batch);
+      const int lc = (int)(rest / batch);  // layer within the call
       // the index words are read before the row count is checked (their slots always exist), so the
       // three small loads are in flight together instead of one after the other
       const int len0 = p.cache_len[b];
@@ -131,6 +137,7 @@ extern "C" int dlm_kv_cache_commit(dlm_ctx* ctx, const dlm_kv_cache* cache, cons
   if (layer_begin < 0 || layer_end > cache->n_layers || layer_begin >= layer_end) return DLM_ERR_SHAPE;
   if ((cache->head_dim * 2) % 16 != 0) return DLM_ERR_UNSUPPORTED;
   if (((uintptr_t)cache->k | (uintptr_t)cache->v | (uintptr_t)k_new | (uintptr_t)v_new) & 15) return DLM_ERR_UNSUPPORTED;
+  DLM_DEVICE_TRY(ctx);
 
   CommitParams p;
   p.cache_k = static_cast<uint4*>(cache->k);
@@ -158,11 +165,27 @@ extern "C" int dlm_kv_cache_commit(dlm_ctx* ctx, const dlm_kv_cache* cache, cons
   p.status = &ctx->words->status;
   p.ticket = &ctx->words->commit_ticket;
 
-  const long long per_block = (long long)kThreads * kUnroll;
-  long long blocks = (p.n_items + per_block - 1) / per_block;
-  const long long max_blocks = (long long)ctx->num_sms * 8;  // 8 resident blocks of 256 threads per SM
+  // one resident wave of equal contiguous ranges; small calls get one block per kThreads * kUnroll items
+  const bool narrow = p.n_items < (1LL << 31) - (long long)kThreads * kUnroll;
+  int& per_sm = ctx->commit_blocks_per_sm[narrow ? 0 : 1];
+  if (per_sm <= 0) {
+    int n = 0;
+    const cudaError_t e = narrow ? cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, kv_commit_kernel<unsigned int>, kThreads, 0)
+                                 : cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, kv_commit_kernel<unsigned long long>, kThreads, 0);
+    if (e != cudaSuccess || n <= 0) return DLM_ERR_CUDA;
+    per_sm = n;
+  }
+  const long long per_pass = (long long)kThreads * kUnroll;
+  long long blocks = (p.n_items + per_pass - 1) / per_pass;
+  const long long max_blocks = (long long)ctx->num_sms * per_sm;
   if (blocks > max_blocks) blocks = max_blocks;
   if (blocks < 1) blocks = 1;
-  DLM_CUDA_TRY(dlm_launch(kv_commit_kernel, dim3((unsigned)blocks), dim3(kThreads), 0, static_cast<cudaStream_t>(stream), p));
+  p.per_block = ((p.n_items + blocks - 1) / blocks + 31) & ~31LL;
+  blocks = (p.n_items + p.per_block - 1) / p.per_block;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  if (narrow)
+    DLM_CUDA_TRY(dlm_launch(kv_commit_kernel<unsigned int>, dim3((unsigned)blocks), dim3(kThreads), 0, st, p));
+  else
+    DLM_CUDA_TRY(dlm_launch(kv_commit_kernel<unsigned long long>, dim3((unsigned)blocks), dim3(kThreads), 0, st, p));
   return dlm_launch_ok(ctx, 1);
 }

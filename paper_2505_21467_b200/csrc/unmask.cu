@@ -307,6 +307,7 @@ extern "C" int dlm_unmask_select(dlm_ctx* ctx, const float* logits, int batch, i
   if (((uintptr_t)logits & 3) != 0) return DLM_ERR_UNSUPPORTED;
   const size_t need = dlm_unmask_workspace_bytes(ctx, batch, block_len, vocab);
   if (!workspace || workspace_bytes < need || ((uintptr_t)workspace & 15)) return DLM_ERR_WORKSPACE;
+  DLM_DEVICE_TRY(ctx);
   unsigned int* tickets = batch <= kDlmUnmaskTickets ? ctx->words->unmask_tickets : nullptr;
   const int n = launch_unmask(logits, batch, block_len, vocab, masked, tokens, k, tok, conf, sel_idx, n_sel,
                               static_cast<Triple*>(workspace), tickets, ctx->num_sms, static_cast<cudaStream_t>(stream));
