@@ -135,3 +135,48 @@ def guided_accept_topk(tok_dlm, tok_ar_topk, masked, tokens, fallback_source=0):
         _p(acc_idx, np.int32), _p(n_acc, np.int32))
     assert rc == 0, rc
     return accept, acc_idx, n_acc
+
+
+def unmask_scores(logits, masked):
+    """Per-position statistics (see oracle.c): returns (tok, conf, zmax, neg_entropy, margin)."""
+    B, Lblk, V = logits.shape
+    tok = np.empty((B, Lblk), np.int32)
+    outs = [np.empty((B, Lblk), np.float32) for _ in range(4)]
+    rc = _load().oracle_unmask_scores(B, Lblk, V, _p(logits, np.float32), _p(masked, np.uint8), _p(tok, np.int32),
+                                      *[_p(o, np.float32) for o in outs])
+    assert rc == 0, rc
+    return (tok, *outs)
+
+
+SCORE_CONFIDENCE, SCORE_NEG_ENTROPY, SCORE_MARGIN, SCORE_LOG_CONF_PLUS_NOISE = 0, 1, 2, 3
+
+
+def unmask_select_scored(logits, masked, tokens, k, kind, noise=None):
+    """Top-k unmasking ranked by the chosen score.  Returns (tok, conf, score, zmax, sel_idx, n_sel)."""
+    B, Lblk, V = logits.shape
+    tok = np.empty((B, Lblk), np.int32)
+    conf, score, zmax = (np.empty((B, Lblk), np.float32) for _ in range(3))
+    sel_idx = np.full((B, max(k, 1)), -1, np.int32) if k > 0 else None
+    n_sel = np.zeros((B,), np.int32) if k > 0 else None
+    rc = _load().oracle_unmask_select_scored(
+        B, Lblk, V, _p(logits, np.float32), _p(masked, np.uint8), _p(tokens, np.int32), k, int(kind),
+        _p(noise, np.float32), _p(tok, np.int32), _p(conf, np.float32), _p(score, np.float32), _p(zmax, np.float32),
+        _p(sel_idx, np.int32), _p(n_sel, np.int32))
+    assert rc == 0, rc
+    return tok, conf, score, zmax, sel_idx, n_sel
+
+
+def guided_accept_threshold(tok_dlm, zmax_dlm, tok_ar_topk, logit_ar_topk, tau, masked, tokens, fallback_source=0):
+    """Top-K match accept plus the confidence threshold of App. C.3.  Returns (accept, acc_idx, n_acc)."""
+    B, Lblk = tok_dlm.shape
+    K = tok_ar_topk.shape[2]
+    assert tok_ar_topk.shape == (B, Lblk, K) == logit_ar_topk.shape and zmax_dlm.shape == (B, Lblk)
+    accept = np.empty((B, Lblk), np.uint8)
+    acc_idx = np.empty((B, Lblk), np.int32)
+    n_acc = np.empty((B,), np.int32)
+    rc = _load().oracle_guided_accept_threshold(
+        B, Lblk, K, _p(tok_dlm, np.int32), _p(zmax_dlm, np.float32), _p(tok_ar_topk, np.int32),
+        _p(logit_ar_topk, np.float32), ctypes.c_float(tau), _p(masked, np.uint8), _p(tokens, np.int32),
+        int(fallback_source), _p(accept, np.uint8), _p(acc_idx, np.int32), _p(n_acc, np.int32))
+    assert rc == 0, rc
+    return accept, acc_idx, n_acc

@@ -321,3 +321,164 @@ int oracle_guided_accept_topk(int B, int Lblk, int K, const int32_t* tok_dlm, co
   }
   return ORACLE_OK;
 }
+
+/*
+ * Per-position statistics for the other ways of choosing U_t that the paper names as baselines
+ * (Sec. 3.1 and the figure on accuracy against the number of denoising steps: a MaskGIT-style sampler, an
+ * entropy-based one and a Top-K margin one).  The paper prints no formula for any of them; the readings taken,
+ * for a masked position with logit row z, p = softmax(z), z_(1) >= z_(2) the two largest entries (a value that
+ * occurs twice counts twice):
+ *     zmax        = z_(1)                                   (the maximum logit)
+ *     conf        = p_(1) = 1 / sum_v exp(z_v - z_(1))      (as in oracle_unmask_select)
+ *     neg_entropy = sum_v p_v log p_v = -(log S - T / S),   S = sum_v exp(z_v - z_(1)), T = sum_v (z_v - z_(1)) exp(z_v - z_(1))
+ *     margin      = p_(1) - p_(2) = (1 - exp(z_(2) - z_(1))) / S        (V == 1: p_(2) = 0)
+ * All sums in fp64, each result rounded once to fp32.  -inf entries contribute nothing (0 * -inf is taken as 0).
+ * Unmasked positions get tok = -1 and -1 in conf; zmax, neg_entropy and margin are written as 0 there.
+ */
+int oracle_unmask_scores(int B, int Lblk, int V, const float* logits, const uint8_t* masked, int32_t* tok,
+                         float* conf, float* zmax, float* neg_entropy, float* margin) {
+#pragma omp parallel for collapse(2) schedule(dynamic, 1)
+  for (int b = 0; b < B; ++b) {
+    for (int i = 0; i < Lblk; ++i) {
+      const size_t p = (size_t)b * Lblk + i;
+      if (!masked[p]) { tok[p] = -1; conf[p] = -1.0f; zmax[p] = 0.f; neg_entropy[p] = 0.f; margin[p] = 0.f; continue; }
+      const float* z = logits + p * (size_t)V;
+      int best = 0;
+      for (int v = 1; v < V; ++v)
+        if (z[v] > z[best]) best = v;
+      double second = -INFINITY; /* largest entry once one occurrence of the maximum is set aside */
+      for (int v = 0; v < V; ++v)
+        if (v != best && (double)z[v] > second) second = (double)z[v];
+      double S = 0.0, T = 0.0;
+      for (int v = 0; v < V; ++v) {
+        const double d = (double)z[v] - (double)z[best];
+        const double e = exp(d);
+        S += e;
+        if (e > 0.0) T += d * e;
+      }
+      tok[p] = best;
+      zmax[p] = z[best];
+      conf[p] = (float)(1.0 / S);
+      neg_entropy[p] = (float)(-(log(S) - T / S));
+      margin[p] = (float)((1.0 - (V > 1 ? exp(second - (double)z[best]) : 0.0)) / S);
+    }
+  }
+  return ORACLE_OK;
+}
+
+/*
+ * Top-k unmasking with a choice of score (the readings above; Eq. 3 still fills with the argmax):
+ *   kind 0  score = conf                            (oracle_unmask_select)
+ *   kind 1  score = neg_entropy                     (entropy-based: most certain distributions first)
+ *   kind 2  score = margin                          (Top-K margin with K = 2)
+ *   kind 3  score = log(conf) + noise[b][i]         (MaskGIT-style: confidence perturbed by noise that the caller
+ *                                                    draws, e.g. temperature * Gumbel; fp64 log, one rounding)
+ * The k_eff = min(k, |M_t|) masked positions of largest score (compared as fp32) are unmasked, ties to the lowest
+ * position; outputs as in oracle_unmask_select plus score [B][Lblk] (-inf... unmasked positions get score 0) and zmax.
+ */
+int oracle_unmask_select_scored(int B, int Lblk, int V, const float* logits, uint8_t* masked, int32_t* tokens, int k,
+                                int kind, const float* noise, int32_t* tok, float* conf, float* score, float* zmax,
+                                int32_t* sel_idx, int32_t* n_sel) {
+  if (kind < 0 || kind > 3 || (kind == 3 && !noise)) return -1;
+  float* ne = (float*)malloc(sizeof(float) * (size_t)B * Lblk);
+  float* mg = (float*)malloc(sizeof(float) * (size_t)B * Lblk);
+  oracle_unmask_scores(B, Lblk, V, logits, masked, tok, conf, zmax, ne, mg);
+  for (size_t p = 0; p < (size_t)B * Lblk; ++p) {
+    if (!masked[p]) { score[p] = 0.f; continue; }
+    if (kind == 0) score[p] = conf[p];
+    else if (kind == 1) score[p] = ne[p];
+    else if (kind == 2) score[p] = mg[p];
+    else score[p] = (float)(log((double)conf[p]) + (double)noise[p]);
+  }
+  free(ne);
+  free(mg);
+  if (k <= 0) return ORACLE_OK;
+  for (int b = 0; b < B; ++b) {
+    uint8_t* mk = masked + (size_t)b * Lblk;
+    const float* sc = score + (size_t)b * Lblk;
+    uint8_t* chosen = (uint8_t*)calloc((size_t)Lblk, 1);
+    int n = 0;
+    for (int round = 0; round < k; ++round) {
+      int best = -1;
+      for (int i = 0; i < Lblk; ++i) {
+        if (!mk[i] || chosen[i]) continue;
+        if (best < 0 || sc[i] > sc[best]) best = i;
+      }
+      if (best < 0) break;
+      chosen[best] = 1;
+      ++n;
+    }
+    int w = 0;
+    for (int i = 0; i < Lblk; ++i) {
+      if (!chosen[i]) continue;
+      sel_idx[(size_t)b * k + w++] = i;
+      tokens[(size_t)b * Lblk + i] = tok[(size_t)b * Lblk + i];
+      mk[i] = 0;
+    }
+    for (; w < k; ++w) sel_idx[(size_t)b * k + w] = -1;
+    n_sel[b] = n;
+    free(chosen);
+  }
+  return ORACLE_OK;
+}
+
+/*
+ * Guided accept with the confidence threshold (App. C.3, "Stochastic Guided Unmasking"; configuration table:
+ * Top-K Assisted Tokens Selection = 2, Guidance Confidence Threshold tau = 0.5).
+ *
+ * The passage says, in short: only the guider's Top-K logits count as guidance logits; besides the deterministic
+ * rule, a token whose largest diffusion logit exceeds tau times the largest guidance logit is unmasked, and
+ * otherwise it stays as it is.  The reading taken:
+ *   1. the deterministic rule is the Top-K match accept above, including its fallback (K = 1: Algorithm 1);
+ *   2. in addition every masked position i with  zmax_dlm[i] > tau * max_j logit_ar_topk[i][j]  is accepted
+ *      (raw logits, as the passage says; the product and the comparison in fp32);
+ *   3. the accepted set is the union, reported in ascending position order; accepted positions receive the DLM
+ *      token, except a position accepted by the fallback alone, which receives the guider's first token when
+ *      fallback_source == 1.
+ * Layouts as oracle_guided_accept_topk, plus zmax_dlm fp32 [B][Lblk] and logit_ar_topk fp32 [B][Lblk][K].
+ */
+int oracle_guided_accept_threshold(int B, int Lblk, int K, const int32_t* tok_dlm, const float* zmax_dlm,
+                                   const int32_t* tok_ar_topk, const float* logit_ar_topk, float tau,
+                                   uint8_t* masked, int32_t* tokens, int fallback_source, uint8_t* accept,
+                                   int32_t* acc_idx, int32_t* n_acc) {
+  if (K <= 0) return -1;
+  for (int b = 0; b < B; ++b) {
+    const size_t o = (size_t)b * Lblk;
+    int first = -1, still_agreeing = 1, n_prefix = 0;
+    for (int i = 0; i < Lblk; ++i) { accept[o + i] = 0; acc_idx[o + i] = -1; }
+    /* 1. deterministic rule: longest prefix of masked positions whose DLM token is among the guider's K */
+    for (int i = 0; i < Lblk; ++i) {
+      if (!masked[o + i]) continue;
+      if (first < 0) first = i;
+      if (!still_agreeing) continue;
+      int among = 0;
+      for (int j = 0; j < K; ++j)
+        if (tok_ar_topk[(o + i) * K + j] == tok_dlm[o + i]) among = 1;
+      if (among) { accept[o + i] = 1; ++n_prefix; } else still_agreeing = 0;
+    }
+    int fallback_pos = -1;
+    if (n_prefix == 0 && first >= 0) { accept[o + first] = 1; fallback_pos = first; }
+    /* 2. threshold rule on every masked position */
+    for (int i = 0; i < Lblk; ++i) {
+      if (!masked[o + i]) continue;
+      float g = logit_ar_topk[(o + i) * K];
+      for (int j = 1; j < K; ++j)
+        if (logit_ar_topk[(o + i) * K + j] > g) g = logit_ar_topk[(o + i) * K + j];
+      const float bound = tau * g;
+      if (zmax_dlm[o + i] > bound) {
+        accept[o + i] = 1;
+        if (i == fallback_pos) fallback_pos = -1; /* accepted in its own right */
+      }
+    }
+    /* 3. union, ascending */
+    int n = 0;
+    for (int i = 0; i < Lblk; ++i) {
+      if (!accept[o + i]) continue;
+      acc_idx[o + n++] = i;
+      tokens[o + i] = (i == fallback_pos && fallback_source == 1) ? tok_ar_topk[(o + i) * K] : tok_dlm[o + i];
+      masked[o + i] = 0;
+    }
+    n_acc[b] = n;
+  }
+  return ORACLE_OK;
+}

@@ -43,3 +43,31 @@ def test_single_rank_needs_no_process_group():
     import bench
     assert bench.max_over_ranks([1.5, 2.5], torch.device("cpu"), 1) == [1.5, 2.5]
     assert bench.job_throughput(1, 64, 8.0) == 8000.0
+
+
+def test_gpus_flag_starts_one_rank_per_gpu(monkeypatch):
+    """`python bench.py --gpus N` outside a launcher starts N ranks itself, the way the launcher would."""
+    sys.path.insert(0, ROOT)
+    import bench
+    seen = {}
+
+    def fake_call(cmd):
+        seen["cmd"] = cmd
+        return 0
+    monkeypatch.setattr(bench.subprocess, "call", fake_call)
+    assert bench.spawn_ranks(4, ["--gpus", "4", "--steps", "8"]) == 0
+    cmd = seen["cmd"]
+    assert cmd[1:4] == ["-m", "torch.distributed.run", "--nnodes=1"]
+    assert "--nproc-per-node=4" in cmd
+    assert cmd[cmd.index("--master-addr") + 1] == "127.0.0.1"
+    assert int(cmd[cmd.index("--master-port") + 1]) > 0
+    assert cmd[-5].endswith("bench.py") and cmd[-4:] == ["--gpus", "4", "--steps", "8"]
+    # and main() takes that path only when no launcher has set the world size
+    monkeypatch.delenv("WORLD_SIZE", raising=False)
+    monkeypatch.setattr(sys, "argv", ["bench.py", "--gpus", "2", "--steps", "4"])
+    monkeypatch.setattr(bench, "spawn_ranks", lambda n, argv: 7 if (n, argv) == (2, ["--gpus", "2", "--steps", "4"]) else 1)
+    try:
+        bench.main()
+        raise AssertionError("main() should exit with the launcher's status")
+    except SystemExit as e:
+        assert e.code == 7
