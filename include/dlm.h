@@ -262,6 +262,57 @@ int dlm_guided_accept_topk(dlm_ctx* ctx, const int32_t* tok_dlm, const int32_t* 
                            int block_len, uint8_t* masked, int32_t* tokens, int fallback_source,
                            uint8_t* accept, int32_t* acc_idx, int32_t* n_acc, void* stream);
 
+/*
+ * dlm_unmask_select_scored — top-k unmasking ranked by a choice of score, all computed in one pass over the
+ * vocabulary (Sec. 3.1 and the figure on accuracy against the number of denoising steps name, as baselines, a
+ * MaskGIT-style sampler, an entropy-based one and a Top-K margin one; Eq. 3 still fills with the argmax).
+ * The paper prints no formula for them.  READINGS taken here (parity is pinned to these readings), for a masked
+ * position with logit row z, p = softmax(z), p_(1) >= p_(2) its two largest entries (a value that occurs twice
+ * counts twice):
+ *   DLM_SCORE_CONFIDENCE           score = p_(1)                               (= dlm_unmask_select)
+ *   DLM_SCORE_NEG_ENTROPY          score = sum_v p_v ln p_v                    (most certain distribution first)
+ *   DLM_SCORE_MARGIN               score = p_(1) - p_(2)                       (Top-K margin with K = 2)
+ *   DLM_SCORE_LOG_CONF_PLUS_NOISE  score = ln p_(1) + noise[b][i]              (MaskGIT-style: the caller draws the
+ *                                   noise, e.g. temperature * Gumbel, so the call itself stays deterministic)
+ * Per batch element the k_eff = min(k, number of masked positions) masked positions of largest score are unmasked,
+ * ties to the lowest position; outputs as dlm_unmask_select, plus
+ *   score  device, fp32 [batch][block_len], out: the ranking score (0 at unmasked positions)
+ *   zmax   device, fp32 [batch][block_len], out: the largest logit of the row (0 at unmasked positions); this is
+ *          the "maximum token logit of the diffusion output" that dlm_guided_accept_threshold takes
+ *   noise  device, fp32 [batch][block_len]; read only for DLM_SCORE_LOG_CONF_PLUS_NOISE, may be NULL otherwise
+ * k == 0 writes tok, conf, score and zmax only.  Workspace from dlm_unmask_scored_workspace_bytes, 16-byte aligned.
+ * Supported: block_len <= 1024.  score_kind outside the four constants is DLM_ERR_SHAPE.
+ */
+enum { DLM_SCORE_CONFIDENCE = 0, DLM_SCORE_NEG_ENTROPY = 1, DLM_SCORE_MARGIN = 2, DLM_SCORE_LOG_CONF_PLUS_NOISE = 3 };
+size_t dlm_unmask_scored_workspace_bytes(const dlm_ctx* ctx, int batch, int block_len, int vocab);
+int dlm_unmask_select_scored(dlm_ctx* ctx, const float* logits, int batch, int block_len, int vocab,
+                             uint8_t* masked, int32_t* tokens, int k, int score_kind, const float* noise,
+                             int32_t* tok, float* conf, float* score, float* zmax, int32_t* sel_idx,
+                             int32_t* n_sel, void* workspace, size_t workspace_bytes, void* stream);
+
+/*
+ * dlm_guided_accept_threshold — the accept rule with the guidance confidence threshold (App. C.3 "Stochastic
+ * Guided Unmasking"; configuration table: Top-K Assisted Tokens Selection = 2, Guidance Confidence Threshold
+ * tau = 0.5).  The passage is short and refers to an "Algorithm 2" that the paper does not contain.  READING taken
+ * (parity is pinned to this reading): the result is the union of
+ *   (1) the deterministic rule: dlm_guided_accept_topk with the same top_k, fallback included, and
+ *   (2) every masked position i with  zmax_dlm[i] > tau * max_j logit_ar_topk[i][j]   (raw logits, as the passage
+ *       says; product and comparison in fp32),
+ * reported in ascending position order.  Accepted positions receive the DLM token; a position accepted by the
+ * fallback alone receives the guider's first token when fallback_source == 1.  The accepted set is in general not
+ * a prefix: commit it with its index list (dlm_kv_cache_commit with src_idx = acc_idx).
+ *
+ *   zmax_dlm       device, fp32 [batch][block_len]: largest DLM logit per position (dlm_unmask_select_scored)
+ *   tok_ar_topk    device, int32 [batch][block_len][top_k], the guider's tokens in rank order
+ *   logit_ar_topk  device, fp32  [batch][block_len][top_k], their logits
+ *   other arguments as dlm_guided_accept_topk.
+ * Supported: block_len <= 1024, 1 <= top_k <= 64; a NaN tau is DLM_ERR_UNSUPPORTED.
+ */
+int dlm_guided_accept_threshold(dlm_ctx* ctx, const int32_t* tok_dlm, const float* zmax_dlm,
+                                const int32_t* tok_ar_topk, const float* logit_ar_topk, int top_k, float tau,
+                                int batch, int block_len, uint8_t* masked, int32_t* tokens, int fallback_source,
+                                uint8_t* accept, int32_t* acc_idx, int32_t* n_acc, void* stream);
+
 #ifdef __cplusplus
 }
 #endif

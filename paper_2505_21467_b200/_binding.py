@@ -67,6 +67,12 @@ def lib() -> ctypes.CDLL:
     L.dlm_unmask_select_static.argtypes = [vp, i32, i32, i32, vp, vp, i32, vp, vp, vp, vp, vp]
     L.dlm_guided_accept.argtypes = [vp, vp, vp, i32, i32, vp, vp, i32, vp, vp, vp, vp]
     L.dlm_guided_accept_topk.argtypes = [vp, vp, vp, i32, i32, i32, vp, vp, i32, vp, vp, vp, vp]
+    L.dlm_unmask_scored_workspace_bytes.argtypes = [vp, i32, i32, i32]
+    L.dlm_unmask_scored_workspace_bytes.restype = sz
+    L.dlm_unmask_select_scored.argtypes = [vp, vp, i32, i32, i32, vp, vp, i32, i32, vp, vp, vp, vp, vp, vp, vp, vp, sz, vp]
+    L.dlm_guided_accept_threshold.argtypes = [vp, vp, vp, vp, vp, i32, f32, i32, i32, vp, vp, i32, vp, vp, vp, vp]
+    for name in ("dlm_unmask_select_scored", "dlm_guided_accept_threshold"):
+        getattr(L, name).restype = i32
     for name in ("dlm_create", "dlm_destroy", "dlm_get_status", "dlm_kv_cache_commit",
                  "dlm_freecache_attn_step", "dlm_unmask_select", "dlm_unmask_select_static", "dlm_guided_accept", "dlm_guided_accept_topk"):
         getattr(L, name).restype = i32
@@ -186,6 +192,32 @@ def dlm_guided_accept_topk(ctx, tok_dlm, tok_ar_topk, top_k, batch, block_len, m
         ctx, _ptr(tok_dlm, torch.int32), _ptr(tok_ar_topk, torch.int32), int(top_k), int(batch), int(block_len),
         _ptr(masked, torch.uint8), _ptr(tokens, torch.int32), int(fallback_source), _ptr(accept, torch.uint8),
         _ptr(acc_idx, torch.int32), _ptr(n_acc, torch.int32), _stream()), "dlm_guided_accept_topk")
+
+
+DLM_SCORE_CONFIDENCE, DLM_SCORE_NEG_ENTROPY, DLM_SCORE_MARGIN, DLM_SCORE_LOG_CONF_PLUS_NOISE = 0, 1, 2, 3
+
+
+def dlm_unmask_scored_workspace_bytes(ctx, batch, block_len, vocab) -> int:
+    return int(lib().dlm_unmask_scored_workspace_bytes(ctx, int(batch), int(block_len), int(vocab)))
+
+
+def dlm_unmask_select_scored(ctx, logits, batch, block_len, vocab, masked, tokens, k, score_kind, noise, tok, conf, score,
+                             zmax, sel_idx, n_sel, workspace) -> None:
+    _check(lib().dlm_unmask_select_scored(
+        ctx, _ptr(logits, torch.float32), int(batch), int(block_len), int(vocab), _ptr(masked, torch.uint8),
+        _ptr(tokens, torch.int32), int(k), int(score_kind), _ptr(noise, torch.float32), _ptr(tok, torch.int32),
+        _ptr(conf, torch.float32), _ptr(score, torch.float32), _ptr(zmax, torch.float32), _ptr(sel_idx, torch.int32),
+        _ptr(n_sel, torch.int32), _ptr(workspace), workspace.numel() * workspace.element_size(), _stream()),
+        "dlm_unmask_select_scored")
+
+
+def dlm_guided_accept_threshold(ctx, tok_dlm, zmax_dlm, tok_ar_topk, logit_ar_topk, top_k, tau, batch, block_len, masked,
+                                tokens, fallback_source, accept, acc_idx, n_acc) -> None:
+    _check(lib().dlm_guided_accept_threshold(
+        ctx, _ptr(tok_dlm, torch.int32), _ptr(zmax_dlm, torch.float32), _ptr(tok_ar_topk, torch.int32),
+        _ptr(logit_ar_topk, torch.float32), int(top_k), float(tau), int(batch), int(block_len), _ptr(masked, torch.uint8),
+        _ptr(tokens, torch.int32), int(fallback_source), _ptr(accept, torch.uint8), _ptr(acc_idx, torch.int32),
+        _ptr(n_acc, torch.int32), _stream()), "dlm_guided_accept_threshold")
 
 
 def dlm_selftest_wait_timeout(ctx, limit_ns: int) -> None:
