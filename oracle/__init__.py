@@ -180,3 +180,29 @@ def guided_accept_threshold(tok_dlm, zmax_dlm, tok_ar_topk, logit_ar_topk, tau, 
         int(fallback_source), _p(accept, np.uint8), _p(acc_idx, np.int32), _p(n_acc, np.int32))
     assert rc == 0, rc
     return accept, acc_idx, n_acc
+
+
+def qkv_project(x, w, bias, Hq, Hkv, D):
+    """x fp32 [B,q_cap,d_model], w fp32 [(Hq+2Hkv)*D, d_model], bias fp32 [(Hq+2Hkv)*D] or None.
+    Returns (q [B,Hq,q_cap,D], k [B,Hkv,q_cap,D], v [B,Hkv,q_cap,D]) fp32."""
+    B, q_cap, d_model = x.shape
+    assert w.shape == ((Hq + 2 * Hkv) * D, d_model)
+    q = np.empty((B, Hq, q_cap, D), np.float32)
+    k = np.empty((B, Hkv, q_cap, D), np.float32)
+    v = np.empty((B, Hkv, q_cap, D), np.float32)
+    rc = _load().oracle_qkv_project(B, q_cap, d_model, Hq, Hkv, D, _p(x, np.float32), _p(w, np.float32),
+                                    _p(bias, np.float32), _p(q, np.float32), _p(k, np.float32), _p(v, np.float32))
+    assert rc == 0, rc
+    return q, k, v
+
+
+def out_project(o, wo, bias):
+    """o fp32 [B,Hq,q_cap,D], wo fp32 [d_model, Hq*D], bias fp32 [d_model] or None.  Returns y fp32 [B,q_cap,d_model]."""
+    B, Hq, q_cap, D = o.shape
+    d_model = wo.shape[0]
+    assert wo.shape == (d_model, Hq * D)
+    y = np.empty((B, q_cap, d_model), np.float32)
+    rc = _load().oracle_out_project(B, q_cap, d_model, Hq, D, _p(o, np.float32), _p(wo, np.float32), _p(bias, np.float32),
+                                    _p(y, np.float32))
+    assert rc == 0, rc
+    return y

@@ -482,3 +482,62 @@ int oracle_guided_accept_threshold(int B, int Lblk, int K, const int32_t* tok_dl
   }
   return ORACLE_OK;
 }
+
+/*
+ * Fused Q/K/V projection of the active window (Table 1 row "Q/K/V projection"; Sec. 3.2.1 "Windowed
+ * Re-computation": the window's K/V are recomputed in every step).
+ *
+ * x is the window's hidden states [B][q_cap][d_model]; w holds the three projection matrices stacked by output
+ * feature, [(Hq + 2 Hkv) * D][d_model] (rows: the Hq query heads, then the Hkv key heads, then the Hkv value heads;
+ * within a head the D features in order), bias [(Hq + 2 Hkv) * D] or NULL.  For output feature n = head * D + d:
+ *     y[b][i][n] = bias[n] + sum_c x[b][i][c] * w[n][c]              (fp64 sum, one rounding to fp32)
+ * and the result is written head by head in the layout the attention step reads:
+ *     q_out [B][Hq][q_cap][D],   k_out, v_out [B][Hkv][q_cap][D].
+ */
+int oracle_qkv_project(int B, int q_cap, int d_model, int Hq, int Hkv, int D, const float* x, const float* w,
+                       const float* bias, float* q_out, float* k_out, float* v_out) {
+  const int n_out = (Hq + 2 * Hkv) * D;
+#pragma omp parallel for collapse(2) schedule(static)
+  for (int b = 0; b < B; ++b) {
+    for (int n = 0; n < n_out; ++n) {
+      const int head = n / D, d = n % D;
+      float* dst;
+      int heads, h;
+      if (head < Hq) { dst = q_out; heads = Hq; h = head; }
+      else if (head < Hq + Hkv) { dst = k_out; heads = Hkv; h = head - Hq; }
+      else { dst = v_out; heads = Hkv; h = head - Hq - Hkv; }
+      for (int i = 0; i < q_cap; ++i) {
+        const float* xr = x + ((size_t)b * q_cap + i) * d_model;
+        const float* wr = w + (size_t)n * d_model;
+        double acc = bias ? (double)bias[n] : 0.0;
+        for (int c = 0; c < d_model; ++c) acc += (double)xr[c] * (double)wr[c];
+        dst[(((size_t)b * heads + h) * q_cap + i) * D + d] = (float)acc;
+      }
+    }
+  }
+  return ORACLE_OK;
+}
+
+/*
+ * Output projection (Table 1 row "output projection"): the attention output [B][Hq][q_cap][D], read with features
+ * ordered (head, d), times wo [d_model][Hq * D]:
+ *     y[b][i][m] = bias[m] + sum_{h,d} o[b][h][i][d] * wo[m][h * D + d]       -> y [B][q_cap][d_model]
+ */
+int oracle_out_project(int B, int q_cap, int d_model, int Hq, int D, const float* o, const float* wo,
+                       const float* bias, float* y) {
+#pragma omp parallel for collapse(2) schedule(static)
+  for (int b = 0; b < B; ++b) {
+    for (int m = 0; m < d_model; ++m) {
+      for (int i = 0; i < q_cap; ++i) {
+        double acc = bias ? (double)bias[m] : 0.0;
+        for (int h = 0; h < Hq; ++h) {
+          const float* orow = o + (((size_t)b * Hq + h) * q_cap + i) * D;
+          const float* wr = wo + (size_t)m * Hq * D + (size_t)h * D;
+          for (int d = 0; d < D; ++d) acc += (double)orow[d] * (double)wr[d];
+        }
+        y[((size_t)b * q_cap + i) * d_model + m] = (float)acc;
+      }
+    }
+  }
+  return ORACLE_OK;
+}
