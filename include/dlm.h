@@ -313,6 +313,39 @@ int dlm_guided_accept_threshold(dlm_ctx* ctx, const int32_t* tok_dlm, const floa
                                 int batch, int block_len, uint8_t* masked, int32_t* tokens, int fallback_source,
                                 uint8_t* accept, int32_t* acc_idx, int32_t* n_acc, void* stream);
 
+/*
+ * dlm_window_qkv_project / dlm_window_out_project — the dense projections either side of the attention step
+ * (Table 1 rows "Q/K/V projection" and "output projection"; Sec. 3.2.1 "Windowed Re-computation": the window's
+ * K/V are recomputed from its hidden states in every step).  bf16 inputs, fp32 accumulation, bf16 outputs.
+ *
+ * dlm_window_qkv_project: for output feature n = head * head_dim + d, with the heads ordered query heads, key
+ * heads, value heads:      y[b][i][n] = bias[n] + sum_c x[b][i][c] * w[n][c]
+ * written head by head in the layout dlm_freecache_attn_step reads, so no transpose sits between the two calls:
+ *   x      device, bf16 [batch][q_cap][d_model]
+ *   w      device, bf16 [(n_q_heads + 2 n_kv_heads) * head_dim][d_model]   (the three matrices stacked by output row)
+ *   bias   device, bf16 [(n_q_heads + 2 n_kv_heads) * head_dim] or NULL
+ *   q_out  device, bf16 [batch][n_q_heads][q_cap][head_dim];  k_out, v_out  bf16 [batch][n_kv_heads][q_cap][head_dim]
+ * Supported: d_model a multiple of 64, (n_q_heads + 2 n_kv_heads) * head_dim a multiple of 128, head_dim a multiple
+ * of 8, 16-byte aligned pointers.
+ *
+ * dlm_window_out_project: y[b][i][m] = bias[m] + sum_{h,d} o[b][h][i][d] * wo[m][h * head_dim + d]
+ *   o      device, bf16 [batch][n_q_heads][q_cap][head_dim]   (the attention step's output, read in place)
+ *   wo     device, bf16 [d_model][n_q_heads * head_dim];  bias bf16 [d_model] or NULL
+ *   y      device, bf16 [batch][q_cap][d_model]
+ * Supported: d_model a multiple of 128, head_dim a multiple of 64, batch * q_cap <= 256, and q_cap a multiple of 8
+ * when batch > 1.
+ *
+ * workspace: device, 256-byte aligned, at least dlm_window_proj_workspace_bytes(ctx, rows = batch * q_cap,
+ * n_out = output features, k_total = contraction length) bytes: fp32 partial tiles of the K split.
+ */
+size_t dlm_window_proj_workspace_bytes(const dlm_ctx* ctx, int rows, int n_out, int k_total);
+int dlm_window_qkv_project(dlm_ctx* ctx, const void* x, const void* w, const void* bias, int batch, int q_cap,
+                           int d_model, int n_q_heads, int n_kv_heads, int head_dim, void* q_out, void* k_out,
+                           void* v_out, void* workspace, size_t workspace_bytes, void* stream);
+int dlm_window_out_project(dlm_ctx* ctx, const void* o, const void* wo, const void* bias, int batch, int q_cap,
+                           int d_model, int n_q_heads, int head_dim, void* y, void* workspace,
+                           size_t workspace_bytes, void* stream);
+
 #ifdef __cplusplus
 }
 #endif

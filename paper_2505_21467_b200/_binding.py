@@ -71,7 +71,11 @@ def lib() -> ctypes.CDLL:
     L.dlm_unmask_scored_workspace_bytes.restype = sz
     L.dlm_unmask_select_scored.argtypes = [vp, vp, i32, i32, i32, vp, vp, i32, i32, vp, vp, vp, vp, vp, vp, vp, vp, sz, vp]
     L.dlm_guided_accept_threshold.argtypes = [vp, vp, vp, vp, vp, i32, f32, i32, i32, vp, vp, i32, vp, vp, vp, vp]
-    for name in ("dlm_unmask_select_scored", "dlm_guided_accept_threshold"):
+    L.dlm_window_proj_workspace_bytes.argtypes = [vp, i32, i32, i32]
+    L.dlm_window_proj_workspace_bytes.restype = sz
+    L.dlm_window_qkv_project.argtypes = [vp, vp, vp, vp, i32, i32, i32, i32, i32, i32, vp, vp, vp, vp, sz, vp]
+    L.dlm_window_out_project.argtypes = [vp, vp, vp, vp, i32, i32, i32, i32, i32, vp, vp, sz, vp]
+    for name in ("dlm_unmask_select_scored", "dlm_guided_accept_threshold", "dlm_window_qkv_project", "dlm_window_out_project"):
         getattr(L, name).restype = i32
     for name in ("dlm_create", "dlm_destroy", "dlm_get_status", "dlm_kv_cache_commit",
                  "dlm_freecache_attn_step", "dlm_unmask_select", "dlm_unmask_select_static", "dlm_guided_accept", "dlm_guided_accept_topk"):
@@ -218,6 +222,26 @@ def dlm_guided_accept_threshold(ctx, tok_dlm, zmax_dlm, tok_ar_topk, logit_ar_to
         _ptr(logit_ar_topk, torch.float32), int(top_k), float(tau), int(batch), int(block_len), _ptr(masked, torch.uint8),
         _ptr(tokens, torch.int32), int(fallback_source), _ptr(accept, torch.uint8), _ptr(acc_idx, torch.int32),
         _ptr(n_acc, torch.int32), _stream()), "dlm_guided_accept_threshold")
+
+
+def dlm_window_proj_workspace_bytes(ctx, rows, n_out, k_total) -> int:
+    return int(lib().dlm_window_proj_workspace_bytes(ctx, int(rows), int(n_out), int(k_total)))
+
+
+def dlm_window_qkv_project(ctx, x, w, bias, batch, q_cap, d_model, n_q_heads, n_kv_heads, head_dim, q_out, k_out, v_out,
+                           workspace) -> None:
+    _check(lib().dlm_window_qkv_project(
+        ctx, _ptr(x, torch.bfloat16), _ptr(w, torch.bfloat16), _ptr(bias, torch.bfloat16), int(batch), int(q_cap), int(d_model),
+        int(n_q_heads), int(n_kv_heads), int(head_dim), _ptr(q_out, torch.bfloat16), _ptr(k_out, torch.bfloat16),
+        _ptr(v_out, torch.bfloat16), _ptr(workspace), workspace.numel() * workspace.element_size(), _stream()),
+        "dlm_window_qkv_project")
+
+
+def dlm_window_out_project(ctx, o, wo, bias, batch, q_cap, d_model, n_q_heads, head_dim, y, workspace) -> None:
+    _check(lib().dlm_window_out_project(
+        ctx, _ptr(o, torch.bfloat16), _ptr(wo, torch.bfloat16), _ptr(bias, torch.bfloat16), int(batch), int(q_cap), int(d_model),
+        int(n_q_heads), int(head_dim), _ptr(y, torch.bfloat16), _ptr(workspace), workspace.numel() * workspace.element_size(),
+        _stream()), "dlm_window_out_project")
 
 
 def dlm_selftest_wait_timeout(ctx, limit_ns: int) -> None:

@@ -24,6 +24,7 @@ extern "C" int dlm_create(dlm_ctx** out, int device) {
   ctx->encode_tiled = nullptr;
   ctx->commit_blocks_per_sm[0] = ctx->commit_blocks_per_sm[1] = 0;
   ctx->attn_smem_limit[0] = ctx->attn_smem_limit[1] = 0;
+  ctx->proj_configured = false;
   if (cudaMalloc(&ctx->words, sizeof(dlm_device_words)) != cudaSuccess ||
       cudaMemset(ctx->words, 0, sizeof(dlm_device_words)) != cudaSuccess) {
     delete ctx;
