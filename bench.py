@@ -605,6 +605,81 @@ def bench_window(name, args, rank, world, local_rank):
                      "algorithmic_bytes_per_launch": kv_bytes + qo_bytes}}))
 
 
+PROJ_CONFIGS = {
+    # name: (base config, d_model, rows per sequence): the window's fused Q/K/V projection and its output projection,
+    # one call per layer over the layers' own weights (so every call streams weights that are not in L2)
+    "dream7b_proj32": ("dream7b", 3584, 32),
+    "dream7b_proj256": ("dream7b", 3584, 256),
+    "llada8b_proj64": ("llada8b", 4096, 64),
+}
+
+
+def bench_proj(name, args, rank, world, local_rank):
+    """Fused Q/K/V projection (and the output projection) of the active window with random weights of the model's
+    widths: a step is one pass over all layers, one call per layer."""
+    base, dm, q_cap = PROJ_CONFIGS[name]
+    cfg = get_config(base)
+    torch.cuda.set_device(local_rank)
+    device = torch.device("cuda", local_rank)
+    import paper_2505_21467_b200 as dlm
+    from paper_2505_21467_b200 import build as _b
+    _b.build()
+    ctx = dlm.dlm_create(device.index)
+    B, NL, Hq, Hkv, D = cfg.batch, cfg.n_layers, cfg.n_q_heads, cfg.n_kv_heads, cfg.head_dim
+    if B * q_cap > 256:
+        B = max(1, 256 // q_cap)
+    n_out = (Hq + 2 * Hkv) * D
+    gen = torch.Generator(device).manual_seed(4242)
+    w = (torch.randn(NL, n_out, dm, generator=gen, device=device) * dm ** -0.5).to(torch.bfloat16)
+    wo = (torch.randn(NL, dm, Hq * D, generator=gen, device=device) * (Hq * D) ** -0.5).to(torch.bfloat16)
+    x = make_kv_rows((B, q_cap, dm), 7, device)
+    q = torch.empty(B, Hq, q_cap, D, dtype=torch.bfloat16, device=device)
+    k = torch.empty(B, Hkv, q_cap, D, dtype=torch.bfloat16, device=device)
+    v = torch.empty_like(k)
+    y = torch.empty(B, q_cap, dm, dtype=torch.bfloat16, device=device)
+    ws = torch.empty(max(dlm.dlm_window_proj_workspace_bytes(ctx, B * q_cap, n_out, dm),
+                         dlm.dlm_window_proj_workspace_bytes(ctx, B * q_cap, dm, Hq * D), 256), dtype=torch.uint8, device=device)
+    sampler = ClockSampler(local_rank)
+    sampler.start()
+    c0 = dlm.dlm_launch_count(ctx)
+    qkv_calls = [(lambda l=l: dlm.dlm_window_qkv_project(ctx, x, w[l], None, B, q_cap, dm, Hq, Hkv, D, q, k, v, ws)) for l in range(NL)]
+    out_calls = [(lambda l=l: dlm.dlm_window_out_project(ctx, q, wo[l], None, B, q_cap, dm, Hq, D, y, ws)) for l in range(NL)]
+    for c in qkv_calls[:3] + out_calls[:3]:
+        c()
+    torch.cuda.synchronize()
+    sampler.mark()
+    t_qkv = time_rotating(qkv_calls, min_launches=NL, replays=max(3, args.steps))
+    t_out = time_rotating(out_calls, min_launches=NL, replays=max(3, args.steps))
+    clocks = sampler.stop()
+    launches = dlm.dlm_launch_count(ctx) - c0
+    status = dlm.dlm_get_status(ctx)
+    if status != 0:
+        raise SystemExit(f"device status {status}: {dlm.dlm_strerror(status)}")
+    peaks = measured_peaks()
+
+    def roof(t, n, kk):
+        rows = B * q_cap
+        nbytes, flops = 2 * (n * kk + rows * kk + rows * n), 2 * rows * n * kk
+        t_b, t_f = nbytes / (peaks["hbm_gbs"] * 1e9), flops / (peaks["bf16_tflops"] * 1e12)
+        bound = "tensor" if t_f > t_b else "hbm"
+        ach, peak = (flops / t / 1e12, peaks["bf16_tflops"]) if bound == "tensor" else (nbytes / t / 1e9, peaks["hbm_gbs"])
+        return {"bound": bound, "achieved": ach, "peak": peak, "unit": "TFLOP/s" if bound == "tensor" else "GB/s", "frac": ach / peak,
+                "peak_source": peaks["source"], "us_per_launch": t * 1e6, "algorithmic_bytes_per_launch": nbytes,
+                "flops_per_launch": flops, "traffic": None}
+    step_s = NL * (t_qkv + t_out)
+    print(json.dumps({
+        "metric": "window_projection_steps_per_s", "value": world / step_s, "unit": "steps/s", "n_gpus": world, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": step_s * 1e3, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "bf16", "data": "synthetic",
+        "config": {"workload": f"{name}: fused Q/K/V projection and output projection of a {B} x {q_cap}-row window, d_model {dm}, "
+                               f"{Hq}q/{Hkv}kv heads x {D}, {NL} layers with their own random weights, one call per layer",
+                   "l2": "every call streams another layer's weights; the layers together are larger than L2",
+                   "launch": "CUDA graph of the C-ABI calls, launches back to back, events around the replays"},
+        "clocks": clocks, "gpu_launches": int(launches),
+        "roofline": dict(kernel="window_proj_kernel (fused Q/K/V projection)", **roof(t_qkv, n_out, dm)),
+        "other_kernels": {"out_projection": roof(t_out, dm, Hq * D)}}))
+
+
 def spawn_ranks(n, argv):
     """`python bench.py --gpus N` outside a launcher: start N ranks on this node, one per GPU, the way the
     launcher would (python -m torch.distributed.run), and pass their output through."""
@@ -630,10 +705,10 @@ def main():
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
-    if args.config in WINDOW_CONFIGS:
+    if args.config in WINDOW_CONFIGS or args.config in PROJ_CONFIGS:
         if args.impl == "reference" or world > 1:
-            raise SystemExit("the window configs run on one GPU with --impl ours")
-        return bench_window(args.config, args, rank, world, local_rank)
+            raise SystemExit("the window and projection configs run on one GPU with --impl ours")
+        return (bench_window if args.config in WINDOW_CONFIGS else bench_proj)(args.config, args, rank, world, local_rank)
     cfg = get_config(args.config)
     cfg_index = ["tiny", "dream7b", "llada8b", "longctx", "guided"].index(cfg.name)
     policy = (f"{cfg.steps_per_block} steps/block, vocab {cfg.vocab}, top-{cfg.top_k}" if cfg.policy == "topk" else

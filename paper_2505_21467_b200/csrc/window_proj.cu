@@ -189,14 +189,10 @@ window_proj_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_consta
       }
       named_bar_sync(1, 128);
     }
-    if (ok && (p.n_split == 1 || *is_last)) {
-      __threadfence();
-      const float bias = p.bias ? __bfloat162float(p.bias[n]) : 0.f;
-      // where this thread's feature goes
-      __nv_bfloat16* dst;
-      size_t row_stride, b_stride;     // elements between consecutive rows of a batch element / between batch elements
+    // where output feature `feat` of row (b, i) goes: element offset of (b = 0, i = 0) and the two strides
+    auto place = [&](int feat, __nv_bfloat16*& dst, size_t& row_stride, size_t& b_stride) {
       if (p.mode == 0) {
-        const int head = n / p.head_dim, d = n % p.head_dim;
+        const int head = feat / p.head_dim, d = feat % p.head_dim;
         int heads, h;
         if (head < p.n_q_heads) { dst = p.q_out; heads = p.n_q_heads; h = head; }
         else if (head < p.n_q_heads + p.n_kv_heads) { dst = p.k_out; heads = p.n_kv_heads; h = head - p.n_q_heads; }
@@ -205,36 +201,60 @@ window_proj_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_consta
         row_stride = p.head_dim;
         b_stride = (size_t)heads * p.q_cap * p.head_dim;
       } else {
-        dst = p.q_out + n;
+        dst = p.q_out + feat;
         row_stride = p.n_out;
         b_stride = (size_t)p.q_cap * p.n_out;
       }
+    };
+    if (ok && p.n_split == 1) {
+      // the whole sum is in TMEM: thread = feature, one 2-byte store per row (the output is small beside the weights)
+      const float bias = p.bias ? __bfloat162float(p.bias[n]) : 0.f;
+      __nv_bfloat16* dst;
+      size_t row_stride, b_stride;
+      place(n, dst, row_stride, b_stride);
       uint32_t v[32];
       for (int c = 0; c < p.rows_pad; c += 32) {
-        float acc[32];
-        if (p.n_split == 1) {
-          tmem_ld32(tmem + ((uint32_t)lane_base << 16) + c, v);
-          tmem_ld_wait();
-#pragma unroll
-          for (int j = 0; j < 32; ++j) acc[j] = __uint_as_float(v[j]);
-        } else {
-#pragma unroll
-          for (int j = 0; j < 32; ++j) acc[j] = 0.f;
-          for (int s2 = 0; s2 < p.n_split; ++s2) {   // fixed order: the sum does not depend on which block came last
-            const float* src = p.partial + (tile_slot + s2) * (size_t)p.rows_pad * kTileN + f;
-#pragma unroll
-            for (int j = 0; j < 32; ++j)
-              if (c + j < rows_here) acc[j] += __ldcg(src + (size_t)(c + j) * kTileN);
-          }
-        }
+        tmem_ld32(tmem + ((uint32_t)lane_base << 16) + c, v);
+        tmem_ld_wait();
 #pragma unroll
         for (int j = 0; j < 32; ++j) {
           const int r = row0 + c + j;
           if (c + j < rows_here) {
             const int b = r / p.q_cap, i = r % p.q_cap;
-            dst[(size_t)b * b_stride + (size_t)i * row_stride] = __float2bfloat16_rn(acc[j] + bias);
+            dst[(size_t)b * b_stride + (size_t)i * row_stride] = __float2bfloat16_rn(__uint_as_float(v[j]) + bias);
           }
         }
+      }
+    } else if (ok && *is_last) {
+      // the last block of the tile adds the partial tiles in split order (the sum does not depend on which block
+      // came last): a thread takes 4 neighbouring features of every fourth row, 16-byte loads, 8-byte stores; a
+      // warp's stores cover 128 features of one row
+      __threadfence();
+      const int t = tid - 64;
+      const int fq = (t & 31) * 4;
+      const int n4 = tile * kTileN + fq;
+      float b4[4] = {0.f, 0.f, 0.f, 0.f};
+      if (p.bias)
+        for (int j = 0; j < 4; ++j) b4[j] = __bfloat162float(p.bias[n4 + j]);
+      __nv_bfloat16* dst;
+      size_t row_stride, b_stride;
+      place(n4, dst, row_stride, b_stride);
+      const float* src0 = p.partial + tile_slot * (size_t)p.rows_pad * kTileN + fq;
+      const size_t split_stride = (size_t)p.rows_pad * kTileN;
+#pragma unroll 4
+      for (int rr = t >> 5; rr < rows_here; rr += 4) {
+        float4 acc = make_float4(b4[0], b4[1], b4[2], b4[3]);
+        for (int s2 = 0; s2 < p.n_split; ++s2) {
+          const float4 x = __ldcg(reinterpret_cast<const float4*>(src0 + s2 * split_stride + (size_t)rr * kTileN));
+          acc.x += x.x; acc.y += x.y; acc.z += x.z; acc.w += x.w;
+        }
+        const int r = row0 + rr;
+        const int b = r / p.q_cap, i = r % p.q_cap;
+        const __nv_bfloat162 lo = __floats2bfloat162_rn(acc.x, acc.y), hi = __floats2bfloat162_rn(acc.z, acc.w);
+        uint2 pk;
+        pk.x = *reinterpret_cast<const uint32_t*>(&lo);
+        pk.y = *reinterpret_cast<const uint32_t*>(&hi);
+        *reinterpret_cast<uint2*>(dst + (size_t)b * b_stride + (size_t)i * row_stride) = pk;
       }
     }
   }
