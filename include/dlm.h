@@ -81,6 +81,14 @@ int64_t dlm_launch_count(const dlm_ctx* ctx);
  * how the give-up path of every wait in the kernels is exercised without hanging a GPU. */
 int dlm_selftest_wait_timeout(dlm_ctx* ctx, uint64_t limit_ns, void* stream);
 
+/* Diagnostic: sets the limit of the attention kernel's device-side waits on work still to come (TMA copies, MMAs,
+ * other blocks' partial results) for the calls that follow; the default is 2 s, the largest value accepted.
+ * 0 means "do not wait at all": the first wait whose data has not arrived yet gives up, every role of the block
+ * unwinds (copies and MMAs already issued are still waited for, with the 2 s limit, before the block releases its
+ * shared memory and TMEM), the kernel ends normally, its outputs are unspecified and dlm_get_status reports
+ * DLM_ERR_TIMEOUT.  This runs the kernel's own give-up path without hanging or faulting anything. */
+int dlm_selftest_set_wait_limit(dlm_ctx* ctx, uint64_t limit_ns);
+
 /* View of a caller-owned KV cache (Sec. 3.2.1: K/V of the prompt and of frozen blocks).
  *   k, v       device, bf16 [n_layers][batch][n_kv_heads][capacity][head_dim]
  *   cache_len  device, int32 [batch]: rows [0, cache_len[b]) are visible to attention.

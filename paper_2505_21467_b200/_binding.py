@@ -53,6 +53,8 @@ def lib() -> ctypes.CDLL:
     L.dlm_strerror.restype = ctypes.c_char_p
     L.dlm_selftest_wait_timeout.argtypes = [vp, ctypes.c_uint64, vp]
     L.dlm_selftest_wait_timeout.restype = i32
+    L.dlm_selftest_set_wait_limit.argtypes = [vp, ctypes.c_uint64]
+    L.dlm_selftest_set_wait_limit.restype = i32
     L.dlm_launch_count.argtypes = [vp]
     L.dlm_launch_count.restype = ctypes.c_int64
     L.dlm_kv_cache_commit.argtypes = [vp, ctypes.POINTER(dlm_kv_cache), vp, vp, i32, vp, vp, i32, vp, i32, i32,
@@ -242,6 +244,10 @@ def dlm_window_out_project(ctx, o, wo, bias, batch, q_cap, d_model, n_q_heads, h
         ctx, _ptr(o, torch.bfloat16), _ptr(wo, torch.bfloat16), _ptr(bias, torch.bfloat16), int(batch), int(q_cap), int(d_model),
         int(n_q_heads), int(head_dim), _ptr(y, torch.bfloat16), _ptr(workspace), workspace.numel() * workspace.element_size(),
         _stream()), "dlm_window_out_project")
+
+
+def dlm_selftest_set_wait_limit(ctx, limit_ns: int) -> None:
+    _check(lib().dlm_selftest_set_wait_limit(ctx, ctypes.c_uint64(int(limit_ns))), "dlm_selftest_set_wait_limit")
 
 
 def dlm_selftest_wait_timeout(ctx, limit_ns: int) -> None:

@@ -25,6 +25,7 @@ extern "C" int dlm_create(dlm_ctx** out, int device) {
   ctx->commit_blocks_per_sm[0] = ctx->commit_blocks_per_sm[1] = 0;
   ctx->attn_smem_limit[0] = ctx->attn_smem_limit[1] = 0;
   ctx->proj_configured = false;
+  ctx->wait_limit_ns = sm100::kWaitLimitNs;
   if (cudaMalloc(&ctx->words, sizeof(dlm_device_words)) != cudaSuccess ||
       cudaMemset(ctx->words, 0, sizeof(dlm_device_words)) != cudaSuccess) {
     delete ctx;
@@ -92,6 +93,13 @@ __global__ void wait_probe_kernel(unsigned long long limit_ns, int* status) {
 }
 
 }  // namespace
+
+extern "C" int dlm_selftest_set_wait_limit(dlm_ctx* ctx, uint64_t limit_ns) {
+  if (!ctx) return DLM_ERR_NULL;
+  if (limit_ns > sm100::kWaitLimitNs) return DLM_ERR_SHAPE;
+  ctx->wait_limit_ns = limit_ns;
+  return DLM_OK;
+}
 
 extern "C" int dlm_selftest_wait_timeout(dlm_ctx* ctx, uint64_t limit_ns, void* stream) {
   if (!ctx) return DLM_ERR_NULL;

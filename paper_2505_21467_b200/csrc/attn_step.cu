@@ -80,6 +80,8 @@ struct AttnParams {
   int fresh_box;   // rows per TMA box of the fresh K/V tensors = min(128, q_cap)
   int whole_units; // 1: deal whole units round-robin, no partials
   int smem_bytes;           // dynamic shared memory of the launch
+  unsigned long long wait_limit_ns;   // limit of every wait of the kernel on work still to come (the context's; 2 s unless
+                                      // a test shortened it); waits that let issued copies and MMAs finish keep 2 s
   float scale_log2;
   int* status;
   unsigned int* tickets;   // one zero-initialised counter per unit: pieces finished
@@ -198,7 +200,8 @@ struct UnitPieces {
 
 // Waits until the counter at `addr` reaches `target` (acquire, device scope).  Bounded like the
 // mbarrier waits: gives up after the same wall-time limit or when the block is aborting.
-__device__ __forceinline__ bool wait_counter(const unsigned int* addr, unsigned int target, volatile int* abort_flag) {
+__device__ __forceinline__ bool wait_counter(const unsigned int* addr, unsigned int target, volatile int* abort_flag,
+                                             uint64_t limit_ns) {
   const uint64_t t0 = global_timer_ns();
   for (uint32_t spin = 1;; ++spin) {
     unsigned int v;
@@ -206,7 +209,7 @@ __device__ __forceinline__ bool wait_counter(const unsigned int* addr, unsigned 
     if (v >= target) return true;
     if ((spin & 15u) == 0u) {
       if (*abort_flag) return false;
-      if (global_timer_ns() - t0 > kWaitLimitNs) {
+      if (global_timer_ns() - t0 > limit_ns) {
         *abort_flag = 1;
         return false;
       }
@@ -445,7 +448,6 @@ attn_step_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
   sched.lc = sched.prefix + p.batch + 1;
   sched.lq = sched.lc + p.batch;
   sched.share_lo = sched.lq + p.batch;
-  int* const merge_slot = sched.share_lo + gridDim.x + 1;   // [grid]
   if (smem_pad + (uint32_t)(p.n_mt + KS + VS) * G::kTileBytes + kBarrierBytes + kFlagBytes +
           4u * (uint32_t)sched_ints(p.batch, gridDim.x) > (uint32_t)p.smem_bytes) {
     // cannot happen with the host's sizing (it leaves room for the largest pad); nothing has been touched yet
@@ -555,13 +557,13 @@ attn_step_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
       if (lane == 0 && has_work) {
         SegmentWalker walk(p, sched, blockIdx.x);
         Segment g;
-        uint32_t kt = 0, vt = 0, seg = 0;
+        uint32_t kt = 0, vt = 0, seg = 0, q_issued = 0;
         bool ok = true;
         while (ok && walk.next(g, n_cta)) {
           if (g.t_end <= g.t_begin) continue;
           const int zq = (g.lc_layer * p.batch + g.b) * p.n_kv_heads + g.kvh;
           const int zc = ((g.lc_layer + p.layer_begin) * p.batch + g.b) * p.n_kv_heads + g.kvh;
-          if (seg > 0) ok = mbar_wait(bar_q_empty, (seg - 1) & 1, abort_ptr);
+          if (seg > 0) ok = mbar_wait_limit(bar_q_empty, (seg - 1) & 1, abort_ptr, p.wait_limit_ns);
           if (!ok) break;
           const int q_box = min(128, p.rows);
           mbar_expect_tx(bar_q_full, (uint32_t)(p.n_mt * q_box) * 128u * G::kPanels);  // a box counts in full
@@ -569,6 +571,7 @@ attn_step_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
             for (int pn = 0; pn < G::kPanels; ++pn)
               tma_load_3d(sm_q + mt * G::kTileBytes + pn * kPanelBytes, &tm_q, bar_q_full, pn * 64,
                           g.rc * p.chunk_rows + mt * 128, zq);
+          ++q_issued;
           for (int t = g.t_begin; t < g.t_end && ok; ++t) {
             const bool cache = t < g.n_ct;
             const int row = cache ? t * kTileKeys : (t - g.n_ct) * p.fresh_box;
@@ -576,7 +579,7 @@ attn_step_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
             const uint32_t bytes = (uint32_t)(cache ? min(kTileKeys, p.capacity) : p.fresh_box) * 128u * G::kPanels;
             {
               const uint32_t s = kt % KS;
-              if (kt >= (uint32_t)KS) ok = mbar_wait(bar_k_empty + 8 * s, ((kt / KS) - 1) & 1, abort_ptr);
+              if (kt >= (uint32_t)KS) ok = mbar_wait_limit(bar_k_empty + 8 * s, ((kt / KS) - 1) & 1, abort_ptr, p.wait_limit_ns);
               if (!ok) break;
               mbar_expect_tx(bar_k_full + 8 * s, bytes);
               for (int pn = 0; pn < G::kPanels; ++pn)
@@ -586,7 +589,7 @@ attn_step_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
             }
             {
               const uint32_t s = vt % VS;
-              if (vt >= (uint32_t)VS) ok = mbar_wait(bar_v_empty + 8 * s, ((vt / VS) - 1) & 1, abort_ptr);
+              if (vt >= (uint32_t)VS) ok = mbar_wait_limit(bar_v_empty + 8 * s, ((vt / VS) - 1) & 1, abort_ptr, p.wait_limit_ns);
               if (!ok) break;
               mbar_expect_tx(bar_v_full + 8 * s, bytes);
               for (int pn = 0; pn < G::kPanels; ++pn)
@@ -603,6 +606,7 @@ attn_step_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
             mbar_wait(bar_k_full + 8 * (i % KS), (i / KS) & 1, never_ptr);
           for (uint32_t i = (vt > (uint32_t)VS ? vt - VS : 0); i < vt; ++i)
             mbar_wait(bar_v_full + 8 * (i % VS), (i / VS) & 1, never_ptr);
+          if (q_issued > 0) mbar_wait(bar_q_full, (q_issued - 1) & 1, never_ptr);
         }
       }
     } else if (warp == 9 || warp == 10) {
@@ -616,7 +620,7 @@ attn_step_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
       const int mt = warp - 9;
       if (has_work && mt < p.n_mt) {
         auto wait_warp = [&](uint32_t bar, uint32_t parity) {
-          return __all_sync(0xffffffffu, mbar_wait(bar, parity, abort_ptr)) != 0;
+          return __all_sync(0xffffffffu, mbar_wait_limit(bar, parity, abort_ptr, p.wait_limit_ns)) != 0;
         };
         SegmentWalker walk(p, sched, blockIdx.x);
         Segment g;
@@ -730,7 +734,7 @@ attn_step_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
         uint32_t pub = 0;
         while (walk.next(g, n_cta)) {
           if (g.slot < 0 || g.merger || g.t_end <= g.t_begin) continue;
-          if (!mbar_wait(bar_pub, pub & 1, abort_ptr)) break;
+          if (!mbar_wait_limit(bar_pub, pub & 1, abort_ptr, p.wait_limit_ns)) break;
           ++pub;
           __threadfence();
           atomicAdd(p.tickets + ((g.lc_layer * p.n_kv_heads + g.kvh) * p.n_rc + g.rc) * p.batch + g.b, 1u);
@@ -751,7 +755,7 @@ attn_step_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
       // the warp leaves a wait together, so the .sync.aligned TMEM instructions that follow
       // always see a converged warp, also when a wait is given up
       auto wait_warp = [&](uint32_t bar, uint32_t parity) {
-        return __all_sync(0xffffffffu, mbar_wait(bar, parity, abort_ptr)) != 0;
+        return __all_sync(0xffffffffu, mbar_wait_limit(bar, parity, abort_ptr, p.wait_limit_ns)) != 0;
       };
       // this thread's query row in row chunk rc of a KV head: which of its query heads, which active row
       auto out_row_of = [&](int lc_layer, int b, int kvh, int rc) {
@@ -893,12 +897,18 @@ attn_step_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
               const int n_others = up.c_last - up.c_first;
               const int unit = ((g.lc_layer * p.n_kv_heads + g.kvh) * p.n_rc + g.rc) * p.batch + g.b;
               if (tid == 0) {
-                *merge_ok = wait_counter(p.tickets + unit, (unsigned int)n_others, abort_ptr) ? 1 : 0;
-                if (*merge_ok) p.tickets[unit] = 0;   // ready for the next launch
+                const bool came = wait_counter(p.tickets + unit, (unsigned int)n_others, abort_ptr, p.wait_limit_ns);
+                if (came) p.tickets[unit] = 0;   // ready for the next launch
+                *merge_ok = came ? 1 : 2;
               }
-              for (int i = tid; i < n_others; i += n_live) merge_slot[i] = up.slot_of(up.c_first + i);
-              named_bar_sync(1, n_live);
-              if (!*merge_ok) { ok = false; break; }
+              // The other threads wait for thread 0's verdict on a flag, not on a hardware barrier: a warp that
+              // gave up earlier never gets here, and a barrier would then wait for it for ever.  Thread 0 always
+              // writes the flag within its own bounded wait; if its warp gave up before, the abort flag is up.
+              for (uint32_t spin = 1; *merge_ok == 0; ++spin)
+                if ((spin & 63u) == 0u && *abort_ptr) break;
+              __syncwarp();
+              const int verdict = __shfl_sync(0xffffffffu, *merge_ok, 0);   // one answer per warp: the code below is .aligned
+              if (verdict != 1) { ok = false; break; }
               __threadfence();
               // maximum and sum over all pieces
               float m_all = m_used, l_all = l_run;
@@ -908,7 +918,7 @@ attn_step_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
                 for (int j = 0; j < 4; ++j)
                   ml[j] = (ib + j < n_others)
                               ? __ldcg(reinterpret_cast<const float2*>(p.ws_ml) +
-                                       ((size_t)merge_slot[ib + j] * p.n_mt + mt) * 128 + row)
+                                       ((size_t)up.slot_of(up.c_first + ib + j) * p.n_mt + mt) * 128 + row)
                               : make_float2(-CUDART_INF_F, 0.f);
                 const float m_new = fmaxf(fmaxf(fmaxf(ml[0].x, ml[1].x), fmaxf(ml[2].x, ml[3].x)), m_all);
                 l_all *= ex2_approx(m_all - m_new);
@@ -923,7 +933,7 @@ attn_step_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
               // O: one other piece at a time, all of its row in flight at once (L2 latency, not
               // bandwidth, bounds a narrower loop); the running sum lives in TMEM between pieces
               for (int i = 0; i < n_others; ++i) {
-                const size_t piece = (size_t)merge_slot[i] * p.n_mt + mt;
+                const size_t piece = (size_t)up.slot_of(up.c_first + i) * p.n_mt + mt;
                 const float4* src = reinterpret_cast<const float4*>(p.ws_o) + piece * (size_t)(D / 4 * 128) + row;
                 float4 x[D / 4];
 #pragma unroll
@@ -1160,6 +1170,7 @@ extern "C" int dlm_freecache_attn_step(dlm_ctx* ctx, const dlm_kv_cache* cache, 
   p.fresh_box = q_cap < 128 ? q_cap : 128;
   p.whole_units = pl.whole_units;
   p.smem_bytes = pl_mut.smem_bytes;
+  p.wait_limit_ns = ctx->wait_limit_ns;
   const float scale = softmax_scale > 0.f ? softmax_scale : 1.0f / sqrtf((float)D);
   p.scale_log2 = scale * 1.4426950408889634f;
   p.status = &ctx->words->status;

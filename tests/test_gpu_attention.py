@@ -227,3 +227,26 @@ def test_a_wait_that_runs_out_reports_timeout_and_leaves_the_context_usable(dev,
     with pytest.raises(dlm.DlmError) as e:
         dlm.dlm_selftest_wait_timeout(dev.ctx, 5_000_000_000)
     assert e.value.code == dlm.DLM_ERR_SHAPE
+
+
+@pytest.mark.parametrize("hint", [1, 0])
+def test_the_attention_kernel_gives_up_cleanly_when_its_waits_may_not_wait(dev, oracle, hint):
+    """The kernel's own unwinding, in both schedules: with the wait limit set to 0 the first wait whose data is still
+    on its way gives up; the producer lets its copies land, the MMA issuers drain, every role reaches the teardown,
+    TMEM is released and the kernel ends normally with DLM_ERR_TIMEOUT.  With the limit restored the next call on the
+    same context is correct again (nothing of the aborted launch is left behind, ticket words included)."""
+    args = dict(NL=2, B=2, Hq=28, Hkv=4, D=128, Lcap=700, q_cap=32, cache_len=[517, 640], seed=4242, hint=hint)
+    dlm.dlm_selftest_set_wait_limit(dev.ctx, 0)
+    try:
+        ck, cv = make_cache(2, 2, 4, 700, 128, 1, device="cuda")
+        q, kn, vn = make_attn_inputs(2, 2, 28, 4, 32, 128, 2, device="cuda")
+        gpu_attn_step(dev, ck, cv, _i32([517, 640]), q, kn, vn, hint=hint)
+        torch.cuda.synchronize()
+        assert dev.status() == dlm.DLM_ERR_TIMEOUT
+    finally:
+        dlm.dlm_selftest_set_wait_limit(dev.ctx, 2_000_000_000)
+    assert dev.status() == 0
+    _case(dev, oracle, **args)
+    with pytest.raises(dlm.DlmError) as e:
+        dlm.dlm_selftest_set_wait_limit(dev.ctx, 3_000_000_000)
+    assert e.value.code == dlm.DLM_ERR_SHAPE
