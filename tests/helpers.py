@@ -10,12 +10,36 @@ ATTN_MEAN_ERR = 2e-3     # mean |err|
 CONF_RTOL = 2e-5         # fp32 confidence: approximate exp and a different summation order
 
 
+GUARD_BYTES = 512
+GUARD_FILL = 0xA5
+
+
 class Dev:
-    """A context plus scratch, created once per test session."""
+    """A context plus scratch, created once per test session.  Output tensors handed out by `guarded` sit between
+    two guard regions of sentinel bytes inside a larger buffer; `status` (which synchronises) checks that no kernel
+    wrote outside its outputs."""
 
     def __init__(self):
         self.ctx = dlm.dlm_create(0)
         self._ws = {}
+        self._guards = []
+
+    def guarded(self, shape, dtype, fill):
+        n = int(np.prod(shape)) * torch.empty((), dtype=dtype).element_size()
+        body = (n + 255) // 256 * 256
+        buf = torch.full((GUARD_BYTES + body + GUARD_BYTES,), GUARD_FILL, dtype=torch.uint8, device="cuda")
+        t = buf[GUARD_BYTES:GUARD_BYTES + n].view(dtype).view(*shape)
+        t.fill_(fill)
+        self._guards.append((buf, n))
+        return t
+
+    def check_guards(self):
+        for buf, n in self._guards:
+            assert bool((buf[:GUARD_BYTES] == GUARD_FILL).all()), "a kernel wrote before the start of an output"
+            assert bool((buf[GUARD_BYTES + n + ((-n) % 256):] == GUARD_FILL).all()) and \
+                bool((buf[GUARD_BYTES + n:GUARD_BYTES + n + ((-n) % 256)] == GUARD_FILL).all()), \
+                "a kernel wrote past the end of an output"
+        self._guards.clear()
 
     def workspace(self, nbytes):
         nbytes = max(int(nbytes), 256)
@@ -25,7 +49,9 @@ class Dev:
         return self._ws[key]
 
     def status(self):
-        return dlm.dlm_get_status(self.ctx)
+        code = dlm.dlm_get_status(self.ctx)     # synchronises the stream
+        self.check_guards()
+        return code
 
 
 def gpu_attn_step(dev, ck, cv, cache_len, q, kn, vn, q_len=None, scale=0.0, layer_begin=0, layer_end=None,
@@ -35,8 +61,8 @@ def gpu_attn_step(dev, ck, cv, cache_len, q, kn, vn, q_len=None, scale=0.0, laye
     nl, _, Hq, q_cap, _ = q.shape
     layer_end = NL if layer_end is None else layer_end
     cache = dlm.make_kv_cache(ck, cv, cache_len)
-    out = torch.full_like(q, float("nan"))
-    lse = torch.full((nl, B, Hq, q_cap), float("nan"), device="cuda") if want_lse else None
+    out = dev.guarded(tuple(q.shape), torch.bfloat16, float("nan"))
+    lse = dev.guarded((nl, B, Hq, q_cap), torch.float32, float("nan")) if want_lse else None
     ws = dev.workspace(dlm.dlm_attn_workspace_bytes(dev.ctx, cache, nl, Hq, q_cap))
     dlm.dlm_freecache_attn_step(dev.ctx, cache, layer_begin, layer_end, q, kn, vn, Hq, q_cap, q_len, scale,
                                 hint, out, lse, ws)
@@ -74,10 +100,10 @@ def assert_attn_close(out_gpu, lse_gpu, ref, lc):
 def gpu_unmask(dev, logits, masked, tokens, k):
     """Runs dlm_unmask_select in place on CUDA tensors; returns (tok, conf, sel_idx, n_sel)."""
     B, Lblk, V = logits.shape
-    tok = torch.full((B, Lblk), -9, dtype=torch.int32, device="cuda")
-    conf = torch.full((B, Lblk), float("nan"), device="cuda")
-    sel_idx = torch.full((B, max(k, 1)), -9, dtype=torch.int32, device="cuda") if k > 0 else None
-    n_sel = torch.full((B,), -9, dtype=torch.int32, device="cuda") if k > 0 else None
+    tok = dev.guarded((B, Lblk), torch.int32, -9)
+    conf = dev.guarded((B, Lblk), torch.float32, float("nan"))
+    sel_idx = dev.guarded((B, max(k, 1)), torch.int32, -9) if k > 0 else None
+    n_sel = dev.guarded((B,), torch.int32, -9) if k > 0 else None
     ws = dev.workspace(dlm.dlm_unmask_workspace_bytes(dev.ctx, B, Lblk, V))
     dlm.dlm_unmask_select(dev.ctx, logits, B, Lblk, V, masked, tokens, k, tok, conf, sel_idx, n_sel, ws)
     return tok, conf, sel_idx, n_sel

@@ -39,7 +39,9 @@ def _run_commit(dev, oracle, ck, cv, cache_len, kn, vn, src_idx=None, dst_pos=No
                                 None if dst_pos is None else np.asarray(dst_pos, np.int32),
                                 None if n_rows is None else np.asarray(n_rows, np.int32), n_max, advance,
                                 layer_begin, layer_end, dst_mode)
-    g_ck, g_cv, g_len = ck.cuda(), cv.cuda(), _i32(cache_len)
+    g_ck = dev.guarded(tuple(ck.shape), torch.bfloat16, 0).copy_(ck)
+    g_cv = dev.guarded(tuple(cv.shape), torch.bfloat16, 0).copy_(cv)
+    g_len = dev.guarded((len(cache_len),), torch.int32, 0).copy_(_i32(cache_len))
     cache = dlm.make_kv_cache(g_ck, g_cv, g_len)
     dlm.dlm_kv_cache_commit(dev.ctx, cache, kn.cuda(), vn.cuda(), src_len, _i32(src_idx), _i32(dst_pos), dst_mode,
                             _i32(n_rows), n_max, advance, layer_begin, layer_end)
@@ -249,9 +251,9 @@ def _compare_guided(dev, oracle, dlm_tok, ar_tok, masked0, source=0):
     o_acc, o_idx, o_n = oracle.guided_accept(dlm_tok, ar_tok, o_masked, o_tokens, source)
     g_masked = torch.from_numpy(masked0.copy()).cuda()
     g_tokens = torch.full((B, Lblk), -4, dtype=torch.int32, device="cuda")
-    accept = torch.full((B, Lblk), 9, dtype=torch.uint8, device="cuda")
-    acc_idx = torch.full((B, Lblk), -9, dtype=torch.int32, device="cuda")
-    n_acc = torch.full((B,), -9, dtype=torch.int32, device="cuda")
+    accept = dev.guarded((B, Lblk), torch.uint8, 9)
+    acc_idx = dev.guarded((B, Lblk), torch.int32, -9)
+    n_acc = dev.guarded((B,), torch.int32, -9)
     dlm.dlm_guided_accept(dev.ctx, torch.from_numpy(dlm_tok).cuda(), torch.from_numpy(ar_tok).cuda(), B, Lblk,
                           g_masked, g_tokens, source, accept, acc_idx, n_acc)
     assert dev.status() == 0
