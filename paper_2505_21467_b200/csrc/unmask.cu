@@ -52,7 +52,7 @@ __device__ __forceinline__ void reduce_chunk(const float* __restrict__ logits, i
   const int chunk = blockIdx.x;
   const float* z = logits + (size_t)row * vocab;
   const int begin = chunk * chunk_len;
-  const int end = min(begin + chunk_len, vocab);
+  const int end = chunk == n_chunks - 1 ? vocab : begin + chunk_len;   // the last chunk takes the remainder (it may be longer)
   const int tid = threadIdx.x;
   constexpr int kStep = kThreads * 4 * U;    // logits per block iteration
 
@@ -143,14 +143,17 @@ __device__ void select_batch(const Triple* partial, int n_chunks, int b, const S
 #pragma unroll
     for (int r = 0; r < RG; ++r) {
       const int i = i0 + r;
-      on[r] = i < L && a.masked[p0 + i] != 0;   // uniform across the warp
+      // the triples are asked for without waiting for the mask byte (a row that is not masked has stale ones,
+      // which are then ignored): one round trip to L2 instead of two in the serial tail of the kernel
+      const uint8_t mk = i < L ? a.masked[p0 + i] : (uint8_t)0;
 #pragma unroll
       for (int h = 0; h < 2; ++h) {
         const int c = lane + 32 * h;
-        v[r][h] = (on[r] && c < n_chunks)
+        v[r][h] = (i < L && c < n_chunks)
                       ? __ldcg(reinterpret_cast<const int4*>(partial + (p0 + i) * n_chunks) + c)
                       : make_int4(__float_as_int(-CUDART_INF_F), 0x7fffffff, 0, 0);
       }
+      on[r] = mk != 0;   // uniform across the warp
     }
 #pragma unroll
     for (int r = 0; r < RG; ++r) {
@@ -273,7 +276,14 @@ int launch_unmask(const float* logits, int batch, int block_len, int vocab, uint
   long long passes = per_block / (2 * 8192);
   passes = passes < 1 ? 1 : (passes > 4 ? 4 : passes);
   const int chunk_len = U * kThreads * 4 * (int)passes;
-  const int n_chunks = (vocab + chunk_len - 1) / chunk_len;
+  int n_chunks = (vocab + chunk_len - 1) / chunk_len;
+  // A short remainder that would push the grid just past one resident wave (Dream's vocabulary at block 32: 19 chunks
+  // x 32 rows = 608 blocks against 592 slots) is folded into the chunk before it: those blocks take a second pass,
+  // which costs less than a second wave in the launch's latency chain.
+  const long long rows = (long long)batch * block_len;
+  if (n_chunks > 1 && rows * n_chunks > wave && rows * (n_chunks - 1) <= wave &&
+      vocab - (long long)(n_chunks - 1) * chunk_len <= chunk_len * 3 / 4)
+    --n_chunks;
   SelectArgs a;
   a.block_len = block_len; a.k = k; a.masked = masked; a.tokens = tokens; a.tok = tok; a.conf = conf;
   a.sel_idx = sel_idx; a.n_sel = n_sel;
