@@ -82,7 +82,8 @@ int64_t dlm_launch_count(const dlm_ctx* ctx);
 int dlm_selftest_wait_timeout(dlm_ctx* ctx, uint64_t limit_ns, void* stream);
 
 /* Diagnostic: sets the limit of the attention kernel's device-side waits on work still to come (TMA copies, MMAs,
- * other blocks' partial results) for the calls that follow; the default is 2 s, the largest value accepted.
+ * other blocks' partial results) for the calls that follow.  Two values are compiled in: 2 000 000 000 (2 s, the
+ * default) and 0; anything else up to 2 s is DLM_ERR_UNSUPPORTED, anything above DLM_ERR_SHAPE.
  * 0 means "do not wait at all": the first wait whose data has not arrived yet gives up, every role of the block
  * unwinds (copies and MMAs already issued are still waited for, with the 2 s limit, before the block releases its
  * shared memory and TMEM), the kernel ends normally, its outputs are unspecified and dlm_get_status reports

@@ -23,7 +23,7 @@ extern "C" int dlm_create(dlm_ctx** out, int device) {
   ctx->launches = 0;
   ctx->encode_tiled = nullptr;
   ctx->commit_blocks_per_sm[0] = ctx->commit_blocks_per_sm[1] = 0;
-  ctx->attn_smem_limit[0] = ctx->attn_smem_limit[1] = 0;
+  for (int i = 0; i < 8; ++i) ctx->attn_smem_limit[i] = 0;
   ctx->proj_configured = false;
   ctx->wait_limit_ns = sm100::kWaitLimitNs;
   if (cudaMalloc(&ctx->words, sizeof(dlm_device_words)) != cudaSuccess ||
@@ -97,6 +97,7 @@ __global__ void wait_probe_kernel(unsigned long long limit_ns, int* status) {
 extern "C" int dlm_selftest_set_wait_limit(dlm_ctx* ctx, uint64_t limit_ns) {
   if (!ctx) return DLM_ERR_NULL;
   if (limit_ns > sm100::kWaitLimitNs) return DLM_ERR_SHAPE;
+  if (limit_ns != 0 && limit_ns != sm100::kWaitLimitNs) return DLM_ERR_UNSUPPORTED;   // the two compiled-in limits
   ctx->wait_limit_ns = limit_ns;
   return DLM_OK;
 }

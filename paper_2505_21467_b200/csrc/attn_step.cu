@@ -47,8 +47,8 @@ constexpr int kTileKeys = 128;
 constexpr int kPanelBytes = 128 * 128;   // one 64-element-wide panel of a 128-row tile
 constexpr int kMaxBatch = 1024;
 constexpr int kTmemCols = 512;
-constexpr int kRegsSoftmax = 208;     // registers per thread of the softmax warpgroups after setmaxnreg.inc
-constexpr int kRegsOther = 88;        // ... of the producer / MMA warpgroup after setmaxnreg.dec
+constexpr int kRegsSoftmax = 216;     // registers per thread of the softmax warpgroups after setmaxnreg.inc
+constexpr int kRegsOther = 72;        // ... of the producer / MMA warpgroup after setmaxnreg.dec
 constexpr int kMaxQCap = 4096;         // active rows per call
 constexpr int kMaxGrid = 256;          // blocks of the persistent grid (one per SM)
 constexpr int kMaxStages = 8;          // barrier slots reserved per ring
@@ -80,8 +80,6 @@ struct AttnParams {
   int fresh_box;   // rows per TMA box of the fresh K/V tensors = min(128, q_cap)
   int whole_units; // 1: deal whole units round-robin, no partials
   int smem_bytes;           // dynamic shared memory of the launch
-  unsigned long long wait_limit_ns;   // limit of every wait of the kernel on work still to come (the context's; 2 s unless
-                                      // a test shortened it); waits that let issued copies and MMAs finish keep 2 s
   float scale_log2;
   int* status;
   unsigned int* tickets;   // one zero-initialised counter per unit: pieces finished
@@ -301,38 +299,26 @@ __device__ __forceinline__ float row_max64(const uint32_t (&s)[64]) {
   return fmaxf(fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3])), fmaxf(fmaxf(mx[4], mx[5]), fmaxf(mx[6], mx[7])));
 }
 
-// Two positive finite floats to a packed pair of bf16 (a in the low half), rounded to nearest with
-// ties away from zero: integer adds and a byte permute.  The conversion instruction runs on the
-// SFU's pipe (2 cycles per warp instruction on top of 8 per exponential), and that pipe is what
-// bounds the softmax warps.
-__device__ __forceinline__ uint32_t pack_bf16_pos(float a, float b) {
-  return __byte_perm(__float_as_uint(a) + 0x8000u, __float_as_uint(b) + 0x8000u, 0x7632);
+__device__ __forceinline__ uint32_t pack_bf16(float a, float b) {
+  const __nv_bfloat162 h = __floats2bfloat162_rn(a, b);
+  return *reinterpret_cast<const uint32_t*>(&h);
 }
 
 // P = 2^(s * scale - m) for 32 scores, packed to bf16 pairs and written to 16 TMEM columns at t_p;
-// adds to the two partial row sums.  The 32 exponentials are independent instructions issued back
-// to back and only then summed and packed: a score-by-score chain (multiply-add, exponential, add)
-// leaves the warp waiting on latencies instead of keeping the SFU busy.
+// adds to the two partial row sums.  (Variants measured in the kernel and found no faster at the
+// configs' shapes: all 32 exponentials issued before the sums, and packing by integer add and byte
+// permute instead of the conversion instruction, which shares the SFU's pipe.)
 __device__ __forceinline__ void exp32_store(const uint32_t* s, float scale_log2, float m_used, uint32_t t_p, float& l0,
                                             float& l1) {
-  float x[32];
-#pragma unroll
-  for (int j = 0; j < 32; ++j) x[j] = fmaf(__uint_as_float(s[j]), scale_log2, -m_used);
-#pragma unroll
-  for (int j = 0; j < 32; ++j) x[j] = ex2_approx(x[j]);
   uint32_t pk[16];
-  float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
 #pragma unroll
-  for (int j = 0; j < 8; ++j) {
-    a0 += x[4 * j];
-    a1 += x[4 * j + 1];
-    a2 += x[4 * j + 2];
-    a3 += x[4 * j + 3];
-    pk[2 * j] = pack_bf16_pos(x[4 * j], x[4 * j + 1]);
-    pk[2 * j + 1] = pack_bf16_pos(x[4 * j + 2], x[4 * j + 3]);
+  for (int j = 0; j < 16; ++j) {
+    const float p0 = ex2_approx(fmaf(__uint_as_float(s[2 * j]), scale_log2, -m_used));
+    const float p1 = ex2_approx(fmaf(__uint_as_float(s[2 * j + 1]), scale_log2, -m_used));
+    l0 += p0;
+    l1 += p1;
+    pk[j] = pack_bf16(p0, p1);
   }
-  l0 += a0 + a2;
-  l1 += a1 + a3;
   tmem_st16(t_p, pk);
 }
 
@@ -409,7 +395,7 @@ __device__ __noinline__ bool softmax_half_ragged(uint32_t t_s, uint32_t t_o, int
       if (c * 32 + 2 * j >= valid) p0 = 0.f;
       if (c * 32 + 2 * j + 1 >= valid) p1 = 0.f;
       l_add += p0 + p1;
-      pk[j] = pack_bf16_pos(p0, p1);
+      pk[j] = pack_bf16(p0, p1);
     }
     tmem_st16(t_s + c * 16, pk);
   }
@@ -418,16 +404,20 @@ __device__ __noinline__ bool softmax_half_ragged(uint32_t t_s, uint32_t t_o, int
   return true;
 }
 
-template <int D>
+// kNoWait = true is the instantiation a test selects to run the give-up path: every wait on work still to come tests
+// its barrier once and gives up if the data is not there yet (waits that let issued copies and MMAs finish keep the
+// 2 s limit).  The limit is a compile-time constant because the waits sit on the critical path of the MMA issuers
+// (a run-time limit cost 2 % at the Dream shape).
+template <int D, int kChunk, bool kNoWait>
 __global__ void __launch_bounds__(kThreads, 1)
 attn_step_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_kc,
                        const __grid_constant__ CUtensorMap tm_vc, const __grid_constant__ CUtensorMap tm_kn,
                        const __grid_constant__ CUtensorMap tm_vn, const AttnParams p) {
   using G = Geometry<D>;
-  // Shared memory of the block, all of it dynamic so that the host can give every byte that is left over
-  // to K/V stages (what bounds this kernel at the configs' shapes is the number of bytes in flight):
-  // [Q: n_mt tiles][K: k_stages tiles][V: v_stages tiles][barriers][flags][scheduling tables], from
-  // the first 1024-byte boundary (the swizzled tiles need that alignment).
+  constexpr uint64_t kLimit = kNoWait ? 0ull : kWaitLimitNs;
+  // Shared memory of the block, all of it dynamic (the scheduling tables are sized by batch and grid):
+  // [Q: n_mt tiles][K ring][V ring][barriers][flags][scheduling tables], from the first 1024-byte
+  // boundary (the swizzled tiles need that alignment).
   extern __shared__ uint8_t smem_raw[];
   // compile-time ring depths: the MMA issuers' scalar code is on the critical path, and divisions by a
   // run-time depth in it cost 10 % at the LLaDA shape
@@ -563,14 +553,14 @@ attn_step_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
           if (g.t_end <= g.t_begin) continue;
           const int zq = (g.lc_layer * p.batch + g.b) * p.n_kv_heads + g.kvh;
           const int zc = ((g.lc_layer + p.layer_begin) * p.batch + g.b) * p.n_kv_heads + g.kvh;
-          if (seg > 0) ok = mbar_wait_limit(bar_q_empty, (seg - 1) & 1, abort_ptr, p.wait_limit_ns);
+          if (seg > 0) ok = mbar_wait_limit(bar_q_empty, (seg - 1) & 1, abort_ptr, kLimit);
           if (!ok) break;
           const int q_box = min(128, p.rows);
           mbar_expect_tx(bar_q_full, (uint32_t)(p.n_mt * q_box) * 128u * G::kPanels);  // a box counts in full
           for (int mt = 0; mt < p.n_mt; ++mt)
             for (int pn = 0; pn < G::kPanels; ++pn)
               tma_load_3d(sm_q + mt * G::kTileBytes + pn * kPanelBytes, &tm_q, bar_q_full, pn * 64,
-                          g.rc * p.chunk_rows + mt * 128, zq);
+                          g.rc * kChunk + mt * 128, zq);
           ++q_issued;
           for (int t = g.t_begin; t < g.t_end && ok; ++t) {
             const bool cache = t < g.n_ct;
@@ -579,7 +569,7 @@ attn_step_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
             const uint32_t bytes = (uint32_t)(cache ? min(kTileKeys, p.capacity) : p.fresh_box) * 128u * G::kPanels;
             {
               const uint32_t s = kt % KS;
-              if (kt >= (uint32_t)KS) ok = mbar_wait_limit(bar_k_empty + 8 * s, ((kt / KS) - 1) & 1, abort_ptr, p.wait_limit_ns);
+              if (kt >= (uint32_t)KS) ok = mbar_wait_limit(bar_k_empty + 8 * s, ((kt / KS) - 1) & 1, abort_ptr, kLimit);
               if (!ok) break;
               mbar_expect_tx(bar_k_full + 8 * s, bytes);
               for (int pn = 0; pn < G::kPanels; ++pn)
@@ -589,7 +579,7 @@ attn_step_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
             }
             {
               const uint32_t s = vt % VS;
-              if (vt >= (uint32_t)VS) ok = mbar_wait_limit(bar_v_empty + 8 * s, ((vt / VS) - 1) & 1, abort_ptr, p.wait_limit_ns);
+              if (vt >= (uint32_t)VS) ok = mbar_wait_limit(bar_v_empty + 8 * s, ((vt / VS) - 1) & 1, abort_ptr, kLimit);
               if (!ok) break;
               mbar_expect_tx(bar_v_full + 8 * s, bytes);
               for (int pn = 0; pn < G::kPanels; ++pn)
@@ -620,7 +610,7 @@ attn_step_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
       const int mt = warp - 9;
       if (has_work && mt < p.n_mt) {
         auto wait_warp = [&](uint32_t bar, uint32_t parity) {
-          return __all_sync(0xffffffffu, mbar_wait_limit(bar, parity, abort_ptr, p.wait_limit_ns)) != 0;
+          return __all_sync(0xffffffffu, mbar_wait_limit(bar, parity, abort_ptr, kLimit)) != 0;
         };
         SegmentWalker walk(p, sched, blockIdx.x);
         Segment g;
@@ -734,7 +724,7 @@ attn_step_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
         uint32_t pub = 0;
         while (walk.next(g, n_cta)) {
           if (g.slot < 0 || g.merger || g.t_end <= g.t_begin) continue;
-          if (!mbar_wait_limit(bar_pub, pub & 1, abort_ptr, p.wait_limit_ns)) break;
+          if (!mbar_wait_limit(bar_pub, pub & 1, abort_ptr, kLimit)) break;
           ++pub;
           __threadfence();
           atomicAdd(p.tickets + ((g.lc_layer * p.n_kv_heads + g.kvh) * p.n_rc + g.rc) * p.batch + g.b, 1u);
@@ -755,11 +745,11 @@ attn_step_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
       // the warp leaves a wait together, so the .sync.aligned TMEM instructions that follow
       // always see a converged warp, also when a wait is given up
       auto wait_warp = [&](uint32_t bar, uint32_t parity) {
-        return __all_sync(0xffffffffu, mbar_wait_limit(bar, parity, abort_ptr, p.wait_limit_ns)) != 0;
+        return __all_sync(0xffffffffu, mbar_wait_limit(bar, parity, abort_ptr, kLimit)) != 0;
       };
       // this thread's query row in row chunk rc of a KV head: which of its query heads, which active row
       auto out_row_of = [&](int lc_layer, int b, int kvh, int rc) {
-        const int r = rc * p.chunk_rows + r_unit;
+        const int r = rc * kChunk + r_unit;
         const int hl = r < p.rows_total ? r / p.q_cap : 0, ir = r < p.rows_total ? r % p.q_cap : 0;
         return (((size_t)lc_layer * p.batch + b) * p.n_q_heads + (size_t)kvh * p.group + hl) * p.q_cap + ir;
       };
@@ -778,7 +768,7 @@ attn_step_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
           const int b = unit % p.batch, grp = unit / p.batch, rc = grp % p.n_rc;
           if (sched.prefix[b + 1] == sched.prefix[b])
             zero_my_row(out_row_of((grp / p.n_rc) / p.n_kv_heads, b, (grp / p.n_rc) % p.n_kv_heads, rc),
-                        rc * p.chunk_rows + r_unit < p.rows_total);
+                        rc * kChunk + r_unit < p.rows_total);
         }
       }
       if (has_work) {
@@ -789,7 +779,7 @@ attn_step_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
         while (ok && walk.next(g, n_cta)) {
           const int n = g.t_end - g.t_begin;
           const size_t qrow = out_row_of(g.lc_layer, g.b, g.kvh, g.rc);
-          const int r_kv = g.rc * p.chunk_rows + r_unit;               // row among all query rows of the KV head
+          const int r_kv = g.rc * kChunk + r_unit;               // row among all query rows of the KV head
           const bool real_row = r_kv < p.rows_total;
           const int i_row = real_row ? r_kv % p.q_cap : 0;
           if (n <= 0) {  // whole-unit mode, inactive batch element: the unit's rows are zero
@@ -897,7 +887,7 @@ attn_step_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
               const int n_others = up.c_last - up.c_first;
               const int unit = ((g.lc_layer * p.n_kv_heads + g.kvh) * p.n_rc + g.rc) * p.batch + g.b;
               if (tid == 0) {
-                const bool came = wait_counter(p.tickets + unit, (unsigned int)n_others, abort_ptr, p.wait_limit_ns);
+                const bool came = wait_counter(p.tickets + unit, (unsigned int)n_others, abort_ptr, kLimit);
                 if (came) p.tickets[unit] = 0;   // ready for the next launch
                 *merge_ok = came ? 1 : 2;
               }
@@ -1021,6 +1011,25 @@ bool register_budget_ok(const cudaFuncAttributes& a) {
   return a.numRegs >= kRegsOther && 8 * (kRegsSoftmax - a.numRegs) <= 4 * (a.numRegs - kRegsOther);
 }
 
+// The eight instantiations: head_dim 128 / 64, row chunks of 256 / 128, normal / no-wait (test) waits.
+using AttnKernel = void (*)(const CUtensorMap, const CUtensorMap, const CUtensorMap, const CUtensorMap, const CUtensorMap,
+                            const AttnParams);
+inline int kernel_index(int head_dim, int chunk_rows, bool no_wait) {
+  return (head_dim == 128 ? 0 : 1) + (chunk_rows == 256 ? 0 : 2) + (no_wait ? 4 : 0);
+}
+AttnKernel kernel_of(int which) {
+  switch (which) {
+    case 0: return attn_step_sm100_kernel<128, 256, false>;
+    case 1: return attn_step_sm100_kernel<64, 256, false>;
+    case 2: return attn_step_sm100_kernel<128, 128, false>;
+    case 3: return attn_step_sm100_kernel<64, 128, false>;
+    case 4: return attn_step_sm100_kernel<128, 256, true>;
+    case 5: return attn_step_sm100_kernel<64, 256, true>;
+    case 6: return attn_step_sm100_kernel<128, 128, true>;
+    default: return attn_step_sm100_kernel<64, 128, true>;
+  }
+}
+
 // First use of an attention kernel on a context's device: checks the register budget and opts in to
 // all the dynamic shared memory the device allows a block (less the kernel's static part).
 int configure_kernel(dlm_ctx* ctx, int which, const void* kern) {
@@ -1135,12 +1144,13 @@ extern "C" int dlm_freecache_attn_step(dlm_ctx* ctx, const dlm_kv_cache* cache, 
   if (!workspace || workspace_bytes < need || ((uintptr_t)workspace & 255)) return DLM_ERR_WORKSPACE;
   const Plan pl = make_plan(ctx, cache, nl, n_q_heads, q_cap, cache_len_hint);
   {
-    const int rc = D == 128 ? configure_kernel(ctx, 0, reinterpret_cast<const void*>(attn_step_sm100_kernel<128>))
-                            : configure_kernel(ctx, 1, reinterpret_cast<const void*>(attn_step_sm100_kernel<64>));
+    const bool nw = ctx->wait_limit_ns == 0;
+    const int which = kernel_index(D, pl.chunk_rows, nw);
+    const int rc = configure_kernel(ctx, which, reinterpret_cast<const void*>(kernel_of(which)));
     if (rc != DLM_OK) return rc;
   }
   Plan pl_mut = pl;
-  if (!plan_shared_memory(ctx->attn_smem_limit[D == 128 ? 0 : 1], D, cache->batch, pl_mut)) return DLM_ERR_UNSUPPORTED;
+  if (!plan_shared_memory(ctx->attn_smem_limit[kernel_index(D, pl.chunk_rows, ctx->wait_limit_ns == 0)], D, cache->batch, pl_mut)) return DLM_ERR_UNSUPPORTED;
   {  // the split schedule counts (unit, key tile) items in 32 bits
     const long long tiles_per_unit = (cache->capacity + 127) / 128 + (q_cap + 127) / 128 + 1;
     if (!pl.whole_units && (long long)nl * cache->batch * cache->n_kv_heads * pl.n_rc * tiles_per_unit >= (1LL << 30))
@@ -1170,7 +1180,6 @@ extern "C" int dlm_freecache_attn_step(dlm_ctx* ctx, const dlm_kv_cache* cache, 
   p.fresh_box = q_cap < 128 ? q_cap : 128;
   p.whole_units = pl.whole_units;
   p.smem_bytes = pl_mut.smem_bytes;
-  p.wait_limit_ns = ctx->wait_limit_ns;
   const float scale = softmax_scale > 0.f ? softmax_scale : 1.0f / sqrtf((float)D);
   p.scale_log2 = scale * 1.4426950408889634f;
   p.status = &ctx->words->status;
@@ -1188,11 +1197,6 @@ extern "C" int dlm_freecache_attn_step(dlm_ctx* ctx, const dlm_kv_cache* cache, 
   if (rc != DLM_OK) return rc;
 
   cudaStream_t s = static_cast<cudaStream_t>(stream);
-  if (D == 128)
-    DLM_CUDA_TRY(dlm_launch(attn_step_sm100_kernel<128>, dim3(pl.grid), dim3(kThreads), (size_t)p.smem_bytes, s, tm_q, tm_kc,
-                            tm_vc, tm_kn, tm_vn, p));
-  else
-    DLM_CUDA_TRY(dlm_launch(attn_step_sm100_kernel<64>, dim3(pl.grid), dim3(kThreads), (size_t)p.smem_bytes, s, tm_q, tm_kc,
-                            tm_vc, tm_kn, tm_vn, p));
+  DLM_CUDA_TRY(dlm_launch(kernel_of(kernel_index(D, pl.chunk_rows, ctx->wait_limit_ns == 0)), dim3(pl.grid), dim3(kThreads), (size_t)p.smem_bytes, s, tm_q, tm_kc, tm_vc, tm_kn, tm_vn, p));
   return dlm_launch_ok(ctx, 1);
 }
