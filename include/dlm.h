@@ -90,6 +90,17 @@ int dlm_selftest_wait_timeout(dlm_ctx* ctx, uint64_t limit_ns, void* stream);
  * DLM_ERR_TIMEOUT.  This runs the kernel's own give-up path without hanging or faulting anything. */
 int dlm_selftest_set_wait_limit(dlm_ctx* ctx, uint64_t limit_ns);
 
+/* Diagnostic: the most blocks (>= 1, else DLM_ERR_SHAPE; unlimited by default, the schedule's own maximum is 16)
+ * that dlm_freecache_attn_step may give one unit in its team schedule, in the calls that follow.  That schedule
+ * serves calls with few (layer, batch element, KV head, row chunk) units: a team of blocks per unit, the unit's
+ * key tiles dealt among them, every block reducing its share of the unit's outputs over all the team's partial
+ * results.  It is chosen when a cost estimate prefers it to the other schedules; force = 1 (0 by default; other
+ * values DLM_ERR_SHAPE) takes it wherever it is possible at all: at most half as many units as SMs and more than
+ * one key tile per unit.  max_blocks = 1 switches the schedule off, so that the same call can be run through the
+ * other schedules and the results compared; they agree to rounding, not bit for bit (the order of the merge
+ * differs). */
+int dlm_selftest_set_attn_team_max(dlm_ctx* ctx, int max_blocks, int force);
+
 /* View of a caller-owned KV cache (Sec. 3.2.1: K/V of the prompt and of frozen blocks).
  *   k, v       device, bf16 [n_layers][batch][n_kv_heads][capacity][head_dim]
  *   cache_len  device, int32 [batch]: rows [0, cache_len[b]) are visible to attention.
@@ -139,6 +150,14 @@ int dlm_kv_cache_commit(dlm_ctx* ctx, const dlm_kv_cache* cache, const void* k_n
  * Returns 0 on invalid arguments. */
 size_t dlm_attn_workspace_bytes(const dlm_ctx* ctx, const dlm_kv_cache* cache,
                                 int n_layers_in_call, int n_q_heads, int q_cap);
+
+/* Diagnostic: the schedule dlm_freecache_attn_step would choose for a call with these arguments (host only,
+ * launches nothing; only the cache's shape fields are read).  Outputs (host): the grid size; the blocks per
+ * team (1 = no teams); whether units are dealt whole (1) or split across blocks (0); query rows per unit
+ * (256 or 128).  DLM_ERR_NULL / DLM_ERR_SHAPE as for the call itself. */
+int dlm_selftest_attn_schedule(const dlm_ctx* ctx, const dlm_kv_cache* cache, int n_layers_in_call, int n_q_heads,
+                               int q_cap, int cache_len_hint, int* grid, int* team, int* whole_units,
+                               int* chunk_rows);
 
 /*
  * dlm_freecache_attn_step — attention of the active window (Sec. 3.2.1 "Windowed

@@ -55,12 +55,17 @@ def lib() -> ctypes.CDLL:
     L.dlm_selftest_wait_timeout.restype = i32
     L.dlm_selftest_set_wait_limit.argtypes = [vp, ctypes.c_uint64]
     L.dlm_selftest_set_wait_limit.restype = i32
+    L.dlm_selftest_set_attn_team_max.argtypes = [vp, ctypes.c_int, ctypes.c_int]
+    L.dlm_selftest_set_attn_team_max.restype = i32
     L.dlm_launch_count.argtypes = [vp]
     L.dlm_launch_count.restype = ctypes.c_int64
     L.dlm_kv_cache_commit.argtypes = [vp, ctypes.POINTER(dlm_kv_cache), vp, vp, i32, vp, vp, i32, vp, i32, i32,
                                       i32, i32, vp]
     L.dlm_attn_workspace_bytes.argtypes = [vp, ctypes.POINTER(dlm_kv_cache), i32, i32, i32]
     L.dlm_attn_workspace_bytes.restype = sz
+    ip = ctypes.POINTER(ctypes.c_int)
+    L.dlm_selftest_attn_schedule.argtypes = [vp, ctypes.POINTER(dlm_kv_cache), i32, i32, i32, i32, ip, ip, ip, ip]
+    L.dlm_selftest_attn_schedule.restype = i32
     L.dlm_freecache_attn_step.argtypes = [vp, ctypes.POINTER(dlm_kv_cache), i32, i32, vp, vp, vp, i32, i32,
                                           vp, f32, i32, vp, vp, vp, sz, vp]
     L.dlm_unmask_workspace_bytes.argtypes = [vp, i32, i32, i32]
@@ -151,6 +156,14 @@ def dlm_kv_cache_commit(ctx, cache, k_new, v_new, src_len, src_idx, dst_pos, dst
 def dlm_attn_workspace_bytes(ctx, cache, n_layers_in_call, n_q_heads, q_cap) -> int:
     return int(lib().dlm_attn_workspace_bytes(ctx, ctypes.byref(cache), int(n_layers_in_call), int(n_q_heads),
                                               int(q_cap)))
+
+
+def dlm_selftest_attn_schedule(ctx, cache, n_layers_in_call, n_q_heads, q_cap, cache_len_hint=0) -> dict:
+    g, c, w, r = ctypes.c_int(), ctypes.c_int(), ctypes.c_int(), ctypes.c_int()
+    _check(lib().dlm_selftest_attn_schedule(ctx, ctypes.byref(cache), int(n_layers_in_call), int(n_q_heads), int(q_cap),
+                                            int(cache_len_hint), ctypes.byref(g), ctypes.byref(c), ctypes.byref(w),
+                                            ctypes.byref(r)), "dlm_selftest_attn_schedule")
+    return {"grid": g.value, "team": c.value, "whole_units": w.value, "chunk_rows": r.value}
 
 
 def dlm_freecache_attn_step(ctx, cache, layer_begin, layer_end, q, k_new, v_new, n_q_heads, q_cap, q_len,
@@ -248,6 +261,10 @@ def dlm_window_out_project(ctx, o, wo, bias, batch, q_cap, d_model, n_q_heads, h
 
 def dlm_selftest_set_wait_limit(ctx, limit_ns: int) -> None:
     _check(lib().dlm_selftest_set_wait_limit(ctx, ctypes.c_uint64(int(limit_ns))), "dlm_selftest_set_wait_limit")
+
+
+def dlm_selftest_set_attn_team_max(ctx, max_blocks: int, force: bool = False) -> None:
+    _check(lib().dlm_selftest_set_attn_team_max(ctx, int(max_blocks), int(force)), "dlm_selftest_set_attn_team_max")
 
 
 def dlm_selftest_wait_timeout(ctx, limit_ns: int) -> None:

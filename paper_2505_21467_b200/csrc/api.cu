@@ -26,6 +26,8 @@ extern "C" int dlm_create(dlm_ctx** out, int device) {
   for (int i = 0; i < 8; ++i) ctx->attn_smem_limit[i] = 0;
   ctx->proj_configured = false;
   ctx->wait_limit_ns = sm100::kWaitLimitNs;
+  ctx->attn_team_max = 1 << 20;   // no limit beyond the schedule's own
+  ctx->attn_team_force = false;
   if (cudaMalloc(&ctx->words, sizeof(dlm_device_words)) != cudaSuccess ||
       cudaMemset(ctx->words, 0, sizeof(dlm_device_words)) != cudaSuccess) {
     delete ctx;
@@ -99,6 +101,14 @@ extern "C" int dlm_selftest_set_wait_limit(dlm_ctx* ctx, uint64_t limit_ns) {
   if (limit_ns > sm100::kWaitLimitNs) return DLM_ERR_SHAPE;
   if (limit_ns != 0 && limit_ns != sm100::kWaitLimitNs) return DLM_ERR_UNSUPPORTED;   // the two compiled-in limits
   ctx->wait_limit_ns = limit_ns;
+  return DLM_OK;
+}
+
+extern "C" int dlm_selftest_set_attn_team_max(dlm_ctx* ctx, int max_blocks, int force) {
+  if (!ctx) return DLM_ERR_NULL;
+  if (max_blocks < 1 || (force != 0 && force != 1)) return DLM_ERR_SHAPE;
+  ctx->attn_team_max = max_blocks;
+  ctx->attn_team_force = force != 0;
   return DLM_OK;
 }
 

@@ -50,6 +50,9 @@ constexpr int kTmemCols = 512;
 constexpr int kRegsSoftmax = 216;     // registers per thread of the softmax warpgroups after setmaxnreg.inc
 constexpr int kRegsOther = 72;        // ... of the producer / MMA warpgroup after setmaxnreg.dec
 constexpr int kMaxQCap = 4096;         // active rows per call
+constexpr double kTeamMergeTiles = 3.0;   // cost of the team schedule's exchange and reduction, in key tiles
+                                          // (measured: about 5 us from the last MMA to the output stores, a key tile 1.7 us)
+constexpr int kTeamMax = 16;              // most blocks of a team
 constexpr int kMaxGrid = 256;          // blocks of the persistent grid (one per SM)
 constexpr int kMaxStages = 8;          // barrier slots reserved per ring
 constexpr int kBarrierBytes = 512;     // mbarriers of a block
@@ -79,6 +82,8 @@ struct AttnParams {
   int n_mt;        // M tiles per unit (1 or 2)
   int fresh_box;   // rows per TMA box of the fresh K/V tensors = min(128, q_cap)
   int whole_units; // 1: deal whole units round-robin, no partials
+  int team;        // > 1 (with whole_units): blocks [u * team, (u + 1) * team) share unit u, key tiles dealt by rank;
+                   // every block then reduces its share of the unit's outputs over all the team's pieces
   int smem_bytes;           // dynamic shared memory of the launch
   float scale_log2;
   int* status;
@@ -98,7 +103,7 @@ struct Segment {
   int lc_layer, b, kvh, rc;   // unit: layer within the call, batch element, KV head, row chunk
   int Lc, Lq, n_ct, T;    // lengths, cache tiles, total tiles of the unit
   int t_begin, t_end;     // tile range of this segment
-  int slot;               // partial slot, or -1 when the segment is the whole unit
+  int slot;               // partial slot; -1 when the segment is the whole unit; -2 for a piece of the team schedule
   int merger;             // partial segment holding the unit's last tile: this block merges the unit
 };
 
@@ -117,7 +122,7 @@ struct SegmentWalker {
   __device__ SegmentWalker(const AttnParams& p_, const Sched& s_, int cta) : p(p_), s(s_) {
     n_units = p.nl * p.n_kv_heads * p.n_rc * p.batch;
     if (p.whole_units) {
-      unit = cta;
+      unit = p.team > 1 ? cta / p.team : cta;
       end = range_begin = 0;
     } else {
       range_begin = s.share_lo[cta];
@@ -141,6 +146,14 @@ struct SegmentWalker {
       g.t_end = g.T;
       g.slot = -1;
       g.merger = 0;
+      if (p.team > 1) {   // this block's share of the unit's key tiles; the launch has one team per unit
+        const int rank = (int)blockIdx.x % p.team;
+        g.t_begin = g.T * rank / p.team;
+        g.t_end = g.T * (rank + 1) / p.team;
+        g.slot = -2;
+        unit = n_units;
+        return true;
+      }
       unit += n_cta;
       return true;
     }
@@ -213,6 +226,162 @@ __device__ __forceinline__ bool wait_counter(const unsigned int* addr, unsigned 
       }
     }
   }
+}
+
+// Team schedule: what a block of a team works on after its share of the key tiles.  The team's pieces lie
+// in the workspace as [rank][M tile][head_dim / 4][128 rows] 16-byte vectors (4 columns of a row) and
+// [rank][M tile][128 rows] (m, l) pairs; the unit's n_mt * head_dim / 4 * 128 output vectors are dealt to
+// the ranks in that storage order, rank r reducing vectors [lo, hi) over all pieces.
+// The launch parameters the team schedule's exchange needs, handed to its functions by value.
+struct TeamArgs {
+  __nv_bfloat16* out;
+  float* lse;
+  float* ws_o;
+  float* ws_ml;
+  unsigned int* tickets;
+  int team, n_mt, batch, n_rc, n_kv_heads, n_q_heads, group, q_cap, rows, rows_total;
+  __device__ explicit TeamArgs(const AttnParams& p)
+      : out(p.out), lse(p.lse), ws_o(p.ws_o), ws_ml(p.ws_ml), tickets(p.tickets), team(p.team), n_mt(p.n_mt),
+        batch(p.batch), n_rc(p.n_rc), n_kv_heads(p.n_kv_heads), n_q_heads(p.n_q_heads), group(p.group), q_cap(p.q_cap),
+        rows(p.rows), rows_total(p.rows_total) {}
+};
+
+struct TeamShare {
+  int rank, unit, b, rc, lc_layer, kvh, lo, hi;
+  bool has_keys;
+  size_t piece0;               // index of the team's first piece
+  uint32_t ml_bytes, o_bytes;  // bytes fetched from each piece: all its (m, l) rows; this block's share of its vectors
+  __device__ TeamShare(const TeamArgs& p, const int* prefix, int D) {
+    const int C = p.team;
+    rank = (int)blockIdx.x % C;
+    unit = (int)blockIdx.x / C;
+    b = unit % p.batch;
+    const int grp = unit / p.batch;
+    rc = grp % p.n_rc;
+    lc_layer = (grp / p.n_rc) / p.n_kv_heads;
+    kvh = (grp / p.n_rc) % p.n_kv_heads;
+    has_keys = prefix[b + 1] > prefix[b];
+    const int n_vec = p.n_mt * (D / 4) * 128;
+    lo = n_vec * rank / C;          // n_vec <= 8192, C <= 16
+    hi = n_vec * (rank + 1) / C;
+    piece0 = (size_t)unit * C * p.n_mt;
+    ml_bytes = (uint32_t)p.n_mt * 128u * 8u;
+    o_bytes = (uint32_t)(hi - lo) * 16u;
+  }
+};
+
+// The two halves of the team schedule's exchange are functions of their own, not inlined: they run once per
+// launch, and inlined they changed the register allocation of the kernel's main loops (measured: 2 - 3 % on the
+// layer-batched calls, which never run them).
+//
+// Publisher warp, one thread: once every softmax thread of this block has stored its row of the block's piece
+// (bar_pub), count the block in the unit's arrival counter; when the whole team has arrived, fetch this
+// block's share of every piece, and every piece's (m, l) rows, into the shared memory the Q, K and V buffers no
+// longer need (all of the block's MMAs have finished by then: every softmax thread waited for its last one).
+// bar_team = bar_pub + 8 completes when all of it has landed.
+template <int D, bool kNoWait>
+__device__ __noinline__ void team_publish(const TeamArgs p, const int* prefix, uint32_t sm_q, uint32_t bar_pub,
+                                          volatile int* abort_ptr) {
+  constexpr uint64_t kLimit = kNoWait ? 0ull : kWaitLimitNs;
+  const uint32_t bar_team = bar_pub + 8;
+  const TeamShare ts(p, prefix, D);
+  if (!ts.has_keys || !mbar_wait_limit(bar_pub, 0, abort_ptr, kLimit)) return;
+  unsigned int* const arrive = p.tickets + ts.unit;
+  unsigned int* const depart = p.tickets + kDlmMaxSplitUnits / 2 + ts.unit;
+  __threadfence();
+  atomicAdd(arrive, 1u);
+  if (!wait_counter(arrive, (unsigned int)p.team, abort_ptr, kLimit)) return;
+  fence_proxy_async_all();
+  mbar_expect_tx(bar_team, (uint32_t)p.team * (ts.ml_bytes + ts.o_bytes));
+  for (int c = 0; c < p.team; ++c) {
+    bulk_load(sm_q + c * ts.ml_bytes, p.ws_ml + (ts.piece0 + (size_t)c * p.n_mt) * 256, ts.ml_bytes, bar_team);
+    bulk_load(sm_q + p.team * ts.ml_bytes + c * ts.o_bytes,
+              p.ws_o + ((ts.piece0 + (size_t)c * p.n_mt) * (size_t)(D / 4 * 128) + ts.lo) * 4, ts.o_bytes, bar_team);
+  }
+  // every block of the team is past its wait on the arrival counter when the last one gets here: the last
+  // one clears both counters for the next launch
+  if (atomicAdd(depart, 1u) == (unsigned int)p.team - 1u) {
+    *arrive = 0;
+    *depart = 0;
+  }
+}
+
+// Softmax threads (all live ones of the block, whole warps): store this thread's row of the block's piece --
+// unnormalised O from TMEM at t_o if the block had key tiles, and (m, l), which is (-inf, 0) if it had none
+// (that piece's O is then never read) -- then wait for the publisher's fetch and reduce this block's share of
+// the unit's output vectors over the C pieces, in rank order.  Returns false when a wait was given up.
+template <int D, int kChunk, bool kNoWait>
+__device__ __noinline__ bool team_exchange(const TeamArgs p, const int* prefix, uint32_t sm_q, uint32_t bar_pub,
+                                           volatile int* abort_ptr, uint32_t t_o, bool has_tiles, float m_used, float l_run) {
+  constexpr uint64_t kLimit = kNoWait ? 0ull : kWaitLimitNs;
+  constexpr int kVecs = D / 4 * 128;          // vectors of one M tile's piece
+  const int tid = threadIdx.x, warp = tid >> 5;
+  const int mt = warp >> 2, row = tid & 127;
+  const int n_live = (p.rows + 31) & ~31;
+  const uint32_t bar_team = bar_pub + 8;
+  const TeamShare ts(p, prefix, D);
+  const int C = p.team;
+  const int Lq = prefix[p.batch + 1 + p.batch + ts.b];   // the clamped q_len table follows the prefix and cache_len tables
+  {
+    const size_t mine = ts.piece0 + (size_t)ts.rank * p.n_mt + mt;
+    if (has_tiles) {
+      float4* po = reinterpret_cast<float4*>(p.ws_o) + mine * (size_t)kVecs + row;
+      uint32_t v[32];
+#pragma unroll 1
+      for (int c = 0; c < D / 32; ++c) {
+        tmem_ld32(t_o + c * 32, v);
+        tmem_ld_wait();
+#pragma unroll
+        for (int j = 0; j < 8; ++j)
+          __stcg(po + (c * 8 + j) * 128, make_float4(__uint_as_float(v[4 * j]), __uint_as_float(v[4 * j + 1]),
+                                                     __uint_as_float(v[4 * j + 2]), __uint_as_float(v[4 * j + 3])));
+      }
+    }
+    __stcg(reinterpret_cast<float2*>(p.ws_ml) + mine * 128 + row, make_float2(m_used, l_run));
+  }
+  __threadfence();
+  mbar_arrive(bar_pub);
+  if (__all_sync(0xffffffffu, mbar_wait_limit(bar_team, 0, abort_ptr, kLimit)) == 0) return false;
+  const uint32_t sm_ml = sm_q, sm_o = sm_q + C * ts.ml_bytes;
+  for (int i = ts.lo + tid; i < ts.hi; i += n_live) {
+    const int mt_i = i / kVecs, rem = i % kVecs, qd = rem / 128, row_i = rem % 128;
+    const int r_unit_i = mt_i * 128 + row_i;
+    const int r_kv_i = ts.rc * kChunk + r_unit_i;
+    if (r_unit_i >= n_live || r_kv_i >= p.rows_total) continue;
+    const int hl = r_kv_i / p.q_cap, ir = r_kv_i % p.q_cap;
+    const size_t qrow_i = (((size_t)ts.lc_layer * p.batch + ts.b) * p.n_q_heads + (size_t)ts.kvh * p.group + hl) * p.q_cap + ir;
+    const bool active_i = ir < Lq;
+    const uint32_t a_ml = sm_ml + (uint32_t)r_unit_i * 8u, a_o = sm_o + (uint32_t)(i - ts.lo) * 16u;
+    float m_all = -CUDART_INF_F;
+#pragma unroll 4
+    for (int c = 0; c < C; ++c) {
+      const float2 ml = ld_shared_f2(a_ml + c * ts.ml_bytes);
+      if (ml.y > 0.f) m_all = fmaxf(m_all, ml.x);
+    }
+    float l_all = 0.f;
+    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll 4
+    for (int c = 0; c < C; ++c) {
+      const float2 ml = ld_shared_f2(a_ml + c * ts.ml_bytes);
+      const float4 x = ld_shared_f4(a_o + c * ts.o_bytes);
+      if (ml.y > 0.f) {   // a piece without keys holds no O
+        const float w = ex2_approx(ml.x - m_all);
+        l_all = fmaf(w, ml.y, l_all);
+        acc.x = fmaf(w, x.x, acc.x);
+        acc.y = fmaf(w, x.y, acc.y);
+        acc.z = fmaf(w, x.z, acc.z);
+        acc.w = fmaf(w, x.w, acc.w);
+      }
+    }
+    const float inv = active_i ? 1.f / l_all : 0.f;
+    const __nv_bfloat162 h0 = __floats2bfloat162_rn(active_i ? acc.x * inv : 0.f, active_i ? acc.y * inv : 0.f);
+    const __nv_bfloat162 h1 = __floats2bfloat162_rn(active_i ? acc.z * inv : 0.f, active_i ? acc.w * inv : 0.f);
+    *reinterpret_cast<uint2*>(p.out + qrow_i * D + qd * 4) =
+        make_uint2(*reinterpret_cast<const uint32_t*>(&h0), *reinterpret_cast<const uint32_t*>(&h1));
+    if (qd == 0 && p.lse) p.lse[qrow_i] = active_i ? (m_all + lg2_approx(l_all)) * 0.6931471805599453f : -CUDART_INF_F;
+  }
+  __syncwarp();
+  return true;
 }
 
 // A key tile is processed in half-steps of up to 64 keys.  Each M tile has two 64-column score
@@ -454,6 +623,7 @@ attn_step_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
                                                                  // products can be in flight, so consecutive half-steps use different
                                                                  // barriers: a parity wait cannot tell phases two apart
   const uint32_t bar_pub = bar_pv_done + 32;                     // partial result of a segment stored by every softmax thread
+  const uint32_t bar_team = bar_pub + 8;                         // team schedule: the team's pieces of this block's share have landed
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   // softmax threads that own a real query row, rounded up to whole warps (they are tid 0 .. n_live-1)
@@ -468,6 +638,7 @@ attn_step_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
     mbar_init(bar_drain, 1);
     mbar_init(bar_drain + 8, 1);
     mbar_init(bar_pub, (uint32_t)n_live);
+    mbar_init(bar_team, 1);
     for (int i = 0; i < KS; ++i) {
       mbar_init(bar_k_full + 8 * i, 1);
       mbar_init(bar_k_empty + 8 * i, (uint32_t)p.n_mt);
@@ -718,7 +889,9 @@ attn_step_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
       // A piece that some other block will merge: once every softmax thread has stored its row
       // (they arrive on bar_pub and move on), make the stores visible device-wide and count the
       // piece in its unit's counter.
-      if (lane == 0 && has_work && !p.whole_units) {
+      if (lane == 0 && p.team > 1) {
+        team_publish<D, kNoWait>(TeamArgs(p), sched.prefix, sm_q, bar_pub, abort_ptr);
+      } else if (lane == 0 && has_work && !p.whole_units) {
         SegmentWalker walk(p, sched, blockIdx.x);
         Segment g;
         uint32_t pub = 0;
@@ -782,8 +955,12 @@ attn_step_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
           const int r_kv = g.rc * kChunk + r_unit;               // row among all query rows of the KV head
           const bool real_row = r_kv < p.rows_total;
           const int i_row = real_row ? r_kv % p.q_cap : 0;
-          if (n <= 0) {  // whole-unit mode, inactive batch element: the unit's rows are zero
-            zero_my_row(qrow, real_row);
+          if (n <= 0) {  // inactive batch element: the unit's rows are zero (team schedule: or no tile for this rank)
+            if (g.T == 0) {
+              zero_my_row(qrow, real_row);
+            } else if (g.slot == -2) {   // a piece without key tiles
+              ok = team_exchange<D, kChunk, kNoWait>(TeamArgs(p), sched.prefix, sm_q, bar_pub, abort_ptr, t_o, false, -CUDART_INF_F, 0.f);
+            }
             continue;
           }
           float m_used = -CUDART_INF_F, l_run = 0.f;
@@ -837,7 +1014,9 @@ attn_step_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
           tc_fence_after_sync();
           const bool active = real_row && i_row < g.Lq;
           uint32_t v[32];
-          if (g.slot < 0) {
+          if (g.slot == -2) {
+            ok = team_exchange<D, kChunk, kNoWait>(TeamArgs(p), sched.prefix, sm_q, bar_pub, abort_ptr, t_o, true, m_used, l_run);
+          } else if (g.slot < 0) {
             const float inv = active ? 1.f / l_run : 0.f;
 #pragma unroll 1
             for (int c = 0; c < D / 32; ++c) {
@@ -1045,7 +1224,7 @@ int configure_kernel(dlm_ctx* ctx, int which, const void* kern) {
 }
 
 struct Plan {
-  int n_mt, rows, rows_total, n_rc, grid, whole_units, chunk_rows;
+  int n_mt, rows, rows_total, n_rc, grid, whole_units, chunk_rows, team;
   int smem_bytes;
   size_t ws_o_bytes, ws_ml_bytes;
 };
@@ -1100,6 +1279,25 @@ Plan make_plan(const dlm_ctx* ctx, const dlm_kv_cache* cache, int nl, int n_q_he
   }
   pl.whole_units = best_shares == 0 ? 1 : 0;
   pl.grid = pl.whole_units ? (int)(units < sms ? units : sms) : best_shares;
+  // Team schedule for calls with few units: C blocks per unit, the unit's key tiles dealt among them, every
+  // block reducing a C-th of the outputs over all pieces in parallel (the split schedule's merging block
+  // folds the other pieces one after the other).  The smallest C that reaches the fewest tiles per block.
+  pl.team = 1;
+  if (ctx->attn_team_max > 1 && may_split && units * 2 <= sms) {
+    long long C = ctx->attn_team_max < kTeamMax ? ctx->attn_team_max : kTeamMax;
+    if (C > sms / units) C = sms / units;
+    if (C > tiles_unit) C = tiles_unit;
+    if (C > 1) {
+      const long long per_block = (tiles_unit + C - 1) / C;
+      C = (tiles_unit + per_block - 1) / per_block;
+      const double t = (double)per_block + kTeamMergeTiles;
+      if (C > 1 && (t < best || ctx->attn_team_force)) {
+        pl.team = (int)C;
+        pl.whole_units = 1;
+        pl.grid = (int)(units * C);
+      }
+    }
+  }
   // the workspace is sized for the split schedule whenever that schedule is possible at all, so
   // that its size does not depend on the hint
   const size_t slots = may_split ? 2 * (size_t)sms : 0;
@@ -1117,6 +1315,21 @@ extern "C" size_t dlm_attn_workspace_bytes(const dlm_ctx* ctx, const dlm_kv_cach
     return 0;
   const Plan pl = make_plan(ctx, cache, n_layers_in_call, n_q_heads, q_cap, 0);
   return pl.ws_o_bytes + pl.ws_ml_bytes + 256;
+}
+
+extern "C" int dlm_selftest_attn_schedule(const dlm_ctx* ctx, const dlm_kv_cache* cache, int n_layers_in_call, int n_q_heads,
+                                          int q_cap, int cache_len_hint, int* grid, int* team, int* whole_units,
+                                          int* chunk_rows) {
+  if (!ctx || !cache || !grid || !team || !whole_units || !chunk_rows) return DLM_ERR_NULL;
+  if (n_layers_in_call <= 0 || n_q_heads <= 0 || q_cap <= 0 || cache->n_kv_heads <= 0 || cache->batch <= 0 ||
+      cache->capacity <= 0 || n_q_heads % cache->n_kv_heads != 0)
+    return DLM_ERR_SHAPE;
+  const Plan pl = make_plan(ctx, cache, n_layers_in_call, n_q_heads, q_cap, cache_len_hint);
+  *grid = pl.grid;
+  *team = pl.team;
+  *whole_units = pl.whole_units;
+  *chunk_rows = pl.chunk_rows;
+  return DLM_OK;
 }
 
 extern "C" int dlm_freecache_attn_step(dlm_ctx* ctx, const dlm_kv_cache* cache, int layer_begin, int layer_end,
@@ -1179,6 +1392,7 @@ extern "C" int dlm_freecache_attn_step(dlm_ctx* ctx, const dlm_kv_cache* cache, 
   p.n_mt = pl.n_mt;
   p.fresh_box = q_cap < 128 ? q_cap : 128;
   p.whole_units = pl.whole_units;
+  p.team = pl.team;
   p.smem_bytes = pl_mut.smem_bytes;
   const float scale = softmax_scale > 0.f ? softmax_scale : 1.0f / sqrtf((float)D);
   p.scale_log2 = scale * 1.4426950408889634f;
@@ -1197,6 +1411,7 @@ extern "C" int dlm_freecache_attn_step(dlm_ctx* ctx, const dlm_kv_cache* cache, 
   if (rc != DLM_OK) return rc;
 
   cudaStream_t s = static_cast<cudaStream_t>(stream);
-  DLM_CUDA_TRY(dlm_launch(kernel_of(kernel_index(D, pl.chunk_rows, ctx->wait_limit_ns == 0)), dim3(pl.grid), dim3(kThreads), (size_t)p.smem_bytes, s, tm_q, tm_kc, tm_vc, tm_kn, tm_vn, p));
+  DLM_CUDA_TRY(dlm_launch(kernel_of(kernel_index(D, pl.chunk_rows, ctx->wait_limit_ns == 0)), dim3(pl.grid), dim3(kThreads),
+                          (size_t)p.smem_bytes, s, tm_q, tm_kc, tm_vc, tm_kn, tm_vn, p));
   return dlm_launch_ok(ctx, 1);
 }

@@ -30,6 +30,8 @@ struct dlm_ctx {
   int commit_blocks_per_sm[2];  // resident blocks per SM of the two commit kernels (0 = not asked yet)
   unsigned long long wait_limit_ns;   // limit of the kernels' device-side waits (2 s; a test may shorten it)
   bool proj_configured;         // shared-memory opt-in of the projection kernel done on this context's device
+  int attn_team_max;            // most blocks the attention call's team schedule may give one unit (1 = schedule off)
+  bool attn_team_force;         // tests: take the team schedule wherever it is possible, whatever the cost estimate says
   int attn_smem_limit[8];       // dynamic shared memory the two attention kernels may use on this device (0 = not set up yet)
 };
 

@@ -250,3 +250,79 @@ def test_the_attention_kernel_gives_up_cleanly_when_its_waits_may_not_wait(dev, 
     with pytest.raises(dlm.DlmError) as e:
         dlm.dlm_selftest_set_wait_limit(dev.ctx, 3_000_000_000)
     assert e.value.code == dlm.DLM_ERR_SHAPE
+
+
+def _schedule(dev, NL, B, Hq, Hkv, D, Lcap, q_cap, nl, hint=0):
+    ck = torch.empty(NL, B, Hkv, Lcap, D, dtype=torch.bfloat16, device="cuda")
+    cache = dlm.make_kv_cache(ck, ck, _i32([0] * B))
+    return dlm.dlm_selftest_attn_schedule(dev.ctx, cache, nl, Hq, q_cap, hint)
+
+
+@pytest.mark.parametrize("NL,B,Hq,Hkv,D,Lcap,q_cap,cache_len,q_len", [
+    (1, 1, 28, 4, 128, 2200, 32, [2048], None),          # one Dream layer at batch 1: 8 units of 128 rows, 17 key tiles each
+    (1, 1, 28, 4, 128, 2200, 32, [2048], [19]),          # ragged active rows
+    (1, 2, 28, 4, 128, 900, 32, [517, 0], [32, 7]),      # an empty cache: one key tile, most ranks get none
+    (1, 2, 6, 2, 128, 700, 20, [256, 255], [20, 0]),     # one element fully inactive; 60 rows per unit
+    (2, 1, 4, 2, 64, 1000, 32, [901], [5]),              # head_dim 64, 64 rows per unit
+    (1, 1, 2, 1, 64, 700, 128, [650], [100]),            # 256 rows per unit (two M tiles), fresh part a whole tile
+    (1, 1, 8, 8, 128, 1100, 64, [1000], None),           # MHA, 64 rows per unit
+    (1, 1, 3, 3, 128, 300, 1, [129], None),              # a single row per unit
+])
+def test_team_schedule_against_the_oracle_at_every_team_size(dev, oracle, NL, B, Hq, Hkv, D, Lcap, q_cap, cache_len, q_len):
+    """Calls with few units give each unit a team of blocks, which split its key tiles and then each reduce a share
+    of its outputs over all the team's pieces.  Every team size, and the same call with the schedule switched off,
+    matches the oracle."""
+    outs = []
+    try:
+        for tmax in (1 << 20, 8, 3, 2, 1):
+            dlm.dlm_selftest_set_attn_team_max(dev.ctx, tmax, force=True)
+            sch = _schedule(dev, NL, B, Hq, Hkv, D, Lcap, q_cap, NL)
+            assert (sch["team"] > 1) == (tmax > 1) and sch["team"] <= tmax and sch["grid"] % sch["team"] == 0
+            out, lse, _ = _case(dev, oracle, NL, B, Hq, Hkv, D, Lcap, q_cap, cache_len, q_len, seed=Hq * 10 + q_cap)
+            outs.append(out.float())
+            if q_len is not None:
+                for b, n in enumerate(q_len):
+                    assert torch.all(out[:, b, :, n:] == 0)
+    finally:
+        dlm.dlm_selftest_set_attn_team_max(dev.ctx, 1 << 20)
+    for o in outs[1:]:
+        assert (o - outs[0]).abs().max().item() <= 2e-2
+    with pytest.raises(dlm.DlmError) as e:
+        dlm.dlm_selftest_set_attn_team_max(dev.ctx, 0)
+    assert e.value.code == dlm.DLM_ERR_SHAPE
+    with pytest.raises(dlm.DlmError) as e:
+        dlm.dlm_selftest_set_attn_team_max(dev.ctx, 4, 2)
+    assert e.value.code == dlm.DLM_ERR_SHAPE
+
+
+def test_team_schedule_repeated_launches_leave_the_counters_clean(dev, oracle):
+    """The team's arrival and departure counters are cleared by the last warp to leave: many launches in a row on
+    the same units (also of different team sizes) stay correct, and so does a split-schedule call afterwards."""
+    shape = dict(NL=1, B=1, Hq=28, Hkv=4, D=128, Lcap=2200, q_cap=32)
+    try:
+        for i, tmax in enumerate((1 << 20, 5, 1 << 20, 2, 9)):
+            dlm.dlm_selftest_set_attn_team_max(dev.ctx, tmax, force=True)
+            assert _schedule(dev, nl=1, **shape)["team"] > 1
+            _case(dev, oracle, cache_len=[1500 + 100 * i], seed=300 + i, **shape)
+    finally:
+        dlm.dlm_selftest_set_attn_team_max(dev.ctx, 1 << 20)
+    _case(dev, oracle, 2, 2, 28, 4, 128, 1400, 32, [1368, 900], [32, 17], seed=77)
+
+
+def test_team_schedule_gives_up_cleanly_when_its_waits_may_not_wait(dev, oracle):
+    """The give-up path under the team schedule: with the wait limit at 0 every wait, the one for the team's other
+    blocks included, gives up at once.  The kernel ends normally with DLM_ERR_TIMEOUT, reading the status clears
+    the half-counted team counters, and the next call is correct."""
+    shape = dict(NL=1, B=1, Hq=28, Hkv=4, D=128, Lcap=2200, q_cap=32)
+    assert _schedule(dev, nl=1, **shape)["team"] > 1
+    dlm.dlm_selftest_set_wait_limit(dev.ctx, 0)
+    try:
+        ck, cv = make_cache(1, 1, 4, 2200, 128, 1, device="cuda")
+        q, kn, vn = make_attn_inputs(1, 1, 28, 4, 32, 128, 2, device="cuda")
+        gpu_attn_step(dev, ck, cv, _i32([2048]), q, kn, vn)
+        torch.cuda.synchronize()
+        assert dev.status() == dlm.DLM_ERR_TIMEOUT
+    finally:
+        dlm.dlm_selftest_set_wait_limit(dev.ctx, 2_000_000_000)
+    assert dev.status() == 0
+    _case(dev, oracle, cache_len=[2048], seed=99, **shape)
