@@ -395,7 +395,11 @@ class Workload:
         with torch.cuda.graph(g, stream=torch.cuda.Stream()):
             layers()
         t = self.time_call(g.replay)
-        return {"us_per_step": t * 1e6, "us_per_layer": t * 1e6 / cfg.n_layers, "calls": cfg.n_layers}
+        sch = dlm.dlm_selftest_attn_schedule(self.ctx, self.cache, 1, cfg.n_q_heads, cfg.block_len, st["cache_len"])
+        return {"us_per_step": t * 1e6, "us_per_layer": t * 1e6 / cfg.n_layers, "calls": cfg.n_layers,
+                "schedule": ("team of %d blocks per unit" % sch["team"]) if sch["team"] > 1 else
+                            ("whole units" if sch["whole_units"] else "units split across blocks"),
+                "grid": sch["grid"], "rows_per_unit": sch["chunk_rows"]}
 
     def other_kernels(self, peak_gbs):
         """HBM-bound kernels of the path, each timed alone: the unmask pass over a fully masked block and the cache

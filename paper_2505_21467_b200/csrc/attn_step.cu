@@ -50,7 +50,7 @@ constexpr int kTmemCols = 512;
 constexpr int kRegsSoftmax = 216;     // registers per thread of the softmax warpgroups after setmaxnreg.inc
 constexpr int kRegsOther = 72;        // ... of the producer / MMA warpgroup after setmaxnreg.dec
 constexpr int kMaxQCap = 4096;         // active rows per call
-constexpr double kTeamMergeTiles = 3.0;   // cost of the team schedule's exchange and reduction, in key tiles
+constexpr double kTeamMergeTiles = 3.0;   // cost of the team schedule's exchange and reduction per M tile, in key tiles
                                           // (measured: about 5 us from the last MMA to the output stores, a key tile 1.7 us)
 constexpr int kTeamMax = 16;              // most blocks of a team
 constexpr int kMaxGrid = 256;          // blocks of the persistent grid (one per SM)
@@ -339,7 +339,8 @@ __device__ __noinline__ bool team_exchange(const TeamArgs p, const int* prefix, 
     }
     __stcg(reinterpret_cast<float2*>(p.ws_ml) + mine * 128 + row, make_float2(m_used, l_run));
   }
-  __threadfence();
+  // no fence here: the arrival below orders the stores before the publisher's wait (block scope), and the
+  // publisher's fence before it counts the block in carries them to device scope
   mbar_arrive(bar_pub);
   if (__all_sync(0xffffffffu, mbar_wait_limit(bar_team, 0, abort_ptr, kLimit)) == 0) return false;
   const uint32_t sm_ml = sm_q, sm_o = sm_q + C * ts.ml_bytes;
@@ -1290,7 +1291,7 @@ Plan make_plan(const dlm_ctx* ctx, const dlm_kv_cache* cache, int nl, int n_q_he
     if (C > 1) {
       const long long per_block = (tiles_unit + C - 1) / C;
       C = (tiles_unit + per_block - 1) / per_block;
-      const double t = (double)per_block + kTeamMergeTiles;
+      const double t = (double)per_block + kTeamMergeTiles * pl.n_mt;   // a piece of two M tiles is twice the bytes
       if (C > 1 && (t < best || ctx->attn_team_force)) {
         pl.team = (int)C;
         pl.whole_units = 1;
