@@ -672,8 +672,23 @@ attn_step_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
     prefetch_tensormap(&tm_vn);
   }
   // everything above needed no data; from here on the inputs of the call are read
+  __syncthreads();   // the barriers exist for the producer's first copy below
   dlm_grid_dependency_wait();
   dlm_trigger_dependents();
+  // Whole units and teams: which unit a block starts with does not depend on the lengths, so the copy of its Q
+  // rows starts now, while the lengths are read and the tile prefix is built (about 1 us, and Q no longer queues
+  // in front of the first K tile).  The roles below consume this Q also when the unit turns out to have no key
+  // tile for this block.
+  const bool early_q = p.whole_units != 0;
+  if (early_q && warp == 8 && lane == 0) {
+    const int unit = p.team > 1 ? (int)blockIdx.x / p.team : (int)blockIdx.x;
+    const int grp = unit / p.batch, b = unit % p.batch, rc = grp % p.n_rc;
+    const int zq = (((grp / p.n_rc) / p.n_kv_heads) * p.batch + b) * p.n_kv_heads + (grp / p.n_rc) % p.n_kv_heads;
+    mbar_expect_tx(bar_q_full, (uint32_t)(p.n_mt * min(128, p.rows)) * 128u * G::kPanels);
+    for (int mt = 0; mt < p.n_mt; ++mt)
+      for (int pn = 0; pn < G::kPanels; ++pn)
+        tma_load_3d(sm_q + mt * G::kTileBytes + pn * kPanelBytes, &tm_q, bar_q_full, pn * 64, rc * kChunk + mt * 128, zq);
+  }
   for (int b = tid; b < p.batch; b += kThreads) {
     int Lc = p.cache_len[b];
     int Lq = p.q_len ? p.q_len[b] : p.q_cap;
@@ -719,21 +734,29 @@ attn_step_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
       if (lane == 0 && has_work) {
         SegmentWalker walk(p, sched, blockIdx.x);
         Segment g;
-        uint32_t kt = 0, vt = 0, seg = 0, q_issued = 0;
+        uint32_t kt = 0, vt = 0, seg = 0, q_issued = early_q ? 1 : 0;
         bool ok = true;
+        bool q_ahead = early_q;   // the Q of the block's first unit is already on its way
         while (ok && walk.next(g, n_cta)) {
-          if (g.t_end <= g.t_begin) continue;
+          const bool q_here = q_ahead;
+          q_ahead = false;
+          if (g.t_end <= g.t_begin) {
+            if (q_here) ++seg;   // the issuers take and release that Q all the same
+            continue;
+          }
           const int zq = (g.lc_layer * p.batch + g.b) * p.n_kv_heads + g.kvh;
           const int zc = ((g.lc_layer + p.layer_begin) * p.batch + g.b) * p.n_kv_heads + g.kvh;
-          if (seg > 0) ok = mbar_wait_limit(bar_q_empty, (seg - 1) & 1, abort_ptr, kLimit);
-          if (!ok) break;
-          const int q_box = min(128, p.rows);
-          mbar_expect_tx(bar_q_full, (uint32_t)(p.n_mt * q_box) * 128u * G::kPanels);  // a box counts in full
-          for (int mt = 0; mt < p.n_mt; ++mt)
-            for (int pn = 0; pn < G::kPanels; ++pn)
-              tma_load_3d(sm_q + mt * G::kTileBytes + pn * kPanelBytes, &tm_q, bar_q_full, pn * 64,
-                          g.rc * kChunk + mt * 128, zq);
-          ++q_issued;
+          if (!q_here) {
+            if (seg > 0) ok = mbar_wait_limit(bar_q_empty, (seg - 1) & 1, abort_ptr, kLimit);
+            if (!ok) break;
+            const int q_box = min(128, p.rows);
+            mbar_expect_tx(bar_q_full, (uint32_t)(p.n_mt * q_box) * 128u * G::kPanels);  // a box counts in full
+            for (int mt = 0; mt < p.n_mt; ++mt)
+              for (int pn = 0; pn < G::kPanels; ++pn)
+                tma_load_3d(sm_q + mt * G::kTileBytes + pn * kPanelBytes, &tm_q, bar_q_full, pn * 64,
+                            g.rc * kChunk + mt * 128, zq);
+            ++q_issued;
+          }
           for (int t = g.t_begin; t < g.t_end && ok; ++t) {
             const bool cache = t < g.n_ct;
             const int row = cache ? t * kTileKeys : (t - g.n_ct) * p.fresh_box;
@@ -830,8 +853,20 @@ attn_step_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
           __syncwarp();
         };
         uint32_t js = 0;   // half-steps whose scores have been issued (global count: buffer = js & 1)
+        bool q_ahead = early_q;   // the Q of the block's first unit was copied before the lengths were known
         while (ok && walk.next(g, n_cta)) {
-          if (g.t_end <= g.t_begin) continue;
+          const bool q_here = q_ahead;
+          q_ahead = false;
+          if (g.t_end <= g.t_begin) {
+            if (q_here) {   // no key tile for this block after all: take that Q and release it
+              ok = wait_warp(bar_q_full, seg & 1);
+              if (!ok) break;
+              if (lane == 0) mbar_arrive(bar_q_empty);
+              __syncwarp();
+              ++seg;
+            }
+            continue;
+          }
           ok = wait_warp(bar_q_full, seg & 1);
           if (!ok) break;
           HalfIter si(g, p.fresh_box), pi(g, p.fresh_box);
