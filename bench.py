@@ -293,29 +293,37 @@ class Workload:
         st = self.sched.at(0)
         self.reset_block_state(st)
         torch.cuda.synchronize()
-        self.graphs = []          # [pool index][last] -> (graph, (e0, e1, e2), kernel launches)
+        # Two graphs per (input set, form of the commit): the step as it is launched, with event nodes only at
+        # its two ends (self.graphs_step: whole-step time), and the same step with one more event node after the
+        # attention launch (self.graphs: the attention launch's own duration; the node costs the step a kernel ->
+        # event -> kernel gap and the overlap of the unmask kernel's prologue with the attention kernel's tail).
+        self.graphs, self.graphs_step = [], []   # [pool index][last] -> (graph, (e0, e1, e2), kernel launches)
         side = torch.cuda.Stream()
         for i in range(self.N_POOL):
             q, kn, vn = self.pool[i]
-            pair = []
+            pair, pair_step = [], []
             for last in (False, True):
-                ev = tuple(torch.cuda.Event(enable_timing=True, external=True) for _ in range(3))
-                g = torch.cuda.CUDAGraph()
-                c0 = dlm.dlm_launch_count(self.ctx)
-                with torch.cuda.graph(g, stream=side):
-                    ev[0].record()
-                    self.launch_attn(st, q, kn, vn)
-                    ev[1].record()
-                    self.launch_rest(last, kn, vn, self.logits[i])
-                    ev[2].record()
-                pair.append((g, ev, dlm.dlm_launch_count(self.ctx) - c0))
+                for with_mid, dest in ((True, pair), (False, pair_step)):
+                    ev = tuple(torch.cuda.Event(enable_timing=True, external=True) for _ in range(3))
+                    g = torch.cuda.CUDAGraph()
+                    c0 = dlm.dlm_launch_count(self.ctx)
+                    with torch.cuda.graph(g, stream=side):
+                        ev[0].record()
+                        self.launch_attn(st, q, kn, vn)
+                        if with_mid:
+                            ev[1].record()
+                        self.launch_rest(last, kn, vn, self.logits[i])
+                        ev[2].record()
+                    dest.append((g, ev, dlm.dlm_launch_count(self.ctx) - c0))
             self.graphs.append(pair)
+            self.graphs_step.append(pair_step)
         torch.cuda.synchronize()
 
-    def run_timed(self, steps):
+    def run_timed(self, steps, attention_events=False):
         """`steps` steps replayed from the graphs; L2 flushed before each; the CUDA events inside the graph bracket
-        the attention call and the whole step on the stream the kernels run on (the flush and the graph's launch
-        latency are outside both).  Returns (total_ms, attn_ms, attn_bytes, attn_flops, kernel launches)."""
+        the whole step (and, with attention_events, the attention call) on the stream the kernels run on (the flush
+        and the graph's launch latency are outside both).  Returns (total_ms, attn_ms, attn_bytes, attn_flops,
+        kernel launches); attn_ms is 0 without attention_events."""
         tot = attn = 0.0
         launches = 0
         nbytes = nflops = 0
@@ -323,12 +331,13 @@ class Workload:
             st = self.sched.at(self.t)
             if st["step_in_block"] == 0:
                 self.reset_block_state(st)
-            g, ev, n = self.graphs[self.t % self.N_POOL][1 if st["last"] else 0]
+            g, ev, n = (self.graphs if attention_events else self.graphs_step)[self.t % self.N_POOL][1 if st["last"] else 0]
             self.flush.zero_()                      # evict L2 between timed steps
             g.replay()
             ev[2].synchronize()
             tot += ev[0].elapsed_time(ev[2])
-            attn += ev[0].elapsed_time(ev[1])
+            if attention_events:
+                attn += ev[0].elapsed_time(ev[1])
             launches += n
             nbytes += attn_bytes(self.cfg, st["cache_len"])
             nflops += attn_flops(self.cfg, st["cache_len"])
@@ -726,7 +735,7 @@ def main():
                           f"{cfg.block_len}, {policy}",
               "attention_launch": "layer-batched (all layers in one call; synthetic stack)",
               "l2": "flushed between timed steps (512 MB write, outside the timed events)",
-              "launch": "each step replayed from one CUDA graph captured from the C-ABI calls, timing events inside the graph", "parallelism": f"replicated x{world} (independent sequences)"}
+              "launch": "each step replayed from one CUDA graph captured from the C-ABI calls, timing event nodes at the two ends of the graph", "parallelism": f"replicated x{world} (independent sequences)"}
 
     if args.impl == "reference":
         if rank != 0:
@@ -774,6 +783,8 @@ def main():
     wl.capture()
     wl.t = 0
     wl.run_timed(max(args.warmup, 3))
+    wl.t = 0
+    wl.run_timed(max(args.warmup, 3), attention_events=True)
     # The timed region: passes of exactly `steps` steps each, repeated until the region has lasted about a
     # second (a single pass of a 60 us step is too short for the clock sampler); the median pass is reported.
     passes = []
@@ -786,7 +797,14 @@ def main():
     barrier()
     clocks = sampler.stop()
     passes.sort(key=lambda r: r[0])
-    tot_ms, attn_ms, nbytes, nflops, launches = passes[len(passes) // 2]
+    tot_ms, _, nbytes, nflops, launches = passes[len(passes) // 2]
+    # the attention launch's own duration: the same steps again, from the graphs that carry an event node after it
+    apasses = []
+    for _ in range(3):
+        wl.t = 0
+        apasses.append(wl.run_timed(args.steps, attention_events=True))
+    apasses.sort(key=lambda r: r[1])
+    tot_attn_ms, attn_ms = apasses[1][0], apasses[1][1]
     status = dlm.dlm_get_status(wl.ctx)
     if status != 0:
         raise SystemExit(f"device status {status}: {dlm.dlm_strerror(status)}")
@@ -803,7 +821,7 @@ def main():
     e2e_steps = min(args.steps, 64)
     e2e_ms = wl.run(e2e_steps, e2e=True, host=host)
 
-    tot_ms, attn_ms, e2e_ms = max_over_ranks([tot_ms, attn_ms, e2e_ms], device, world)
+    tot_ms, attn_ms, e2e_ms, tot_attn_ms = max_over_ranks([tot_ms, attn_ms, e2e_ms, tot_attn_ms], device, world)
     if rank != 0:
         if world > 1:
             dist.destroy_process_group()
@@ -825,7 +843,9 @@ def main():
         "roofline": {"kernel": "attention step (all layers, one launch)", "bound": bound, "achieved": ach,
                      "peak": peak, "unit": "TFLOP/s" if bound == "tensor" else "GB/s", "frac": ach / peak,
                      "peak_source": peaks["source"], "traffic": ATTN_DRAM_TRAFFIC_BYTES.get(cfg.name),
-                     "protocol": "events inside the step graph around the attention launch, L2 flushed before the step",
+                     "protocol": "events inside the step graph around the attention launch, L2 flushed before the step; a pass of "
+                                 "its own over the same steps, because the event node after the launch lengthens the step",
+                     "ms_per_step_with_that_event": tot_attn_ms / args.steps,
                      "attn_us_per_launch": attn_ms * 1e3 / args.steps,
                      "attn_tflops": nflops / attn_s / 1e12, "attn_GB/s": nbytes / attn_s / 1e9,
                      "frac_of_bytes_roof": t_bytes / attn_s, "frac_of_flops_roof": t_flops / attn_s,
