@@ -40,8 +40,8 @@ from workloads import (get_config, make_attn_inputs, make_cache, make_kv_rows, m
 # attention kernel as it stands (see profiles/).  A workload without a capture, or whose capture predates a
 # change of the kernel, has no entry and the line prints null.
 ATTN_DRAM_TRAFFIC_BYTES = {
-    "dream7b": 68.5e6,             # 67.07 MB read + 1.45 MB written (profiles/attn_step_sm100_dream7b.md)
-    "dream7b_window256": 231.6e6,   # 182.2 MB read + 49.4 MB written (profiles/attn_step_sm100_window256.md)
+    "dream7b": 68.7e6,             # 67.08 MB read + 1.6 MB written (profiles/attn_step_sm100_dream7b.md)
+    "dream7b_window256": 226.5e6,   # 176.9 MB read + 49.6 MB written, the lower of two launches (profiles/attn_step_sm100_window256.md)
 }
 
 L2_BYTES = 126 << 20
