@@ -196,6 +196,21 @@ def qkv_project(x, w, bias, Hq, Hkv, D):
     return q, k, v
 
 
+def qkv_project_rope(x, w, bias, rope_cos, rope_sin, Hq, Hkv, D):
+    """qkv_project followed by the rotary embedding of the query and key heads (half-split pairs d, d + D/2);
+    rope_cos, rope_sin fp32 [B,q_cap,D/2].  Returns (q, k, v) like qkv_project."""
+    B, q_cap, d_model = x.shape
+    assert w.shape == ((Hq + 2 * Hkv) * D, d_model) and rope_cos.shape == (B, q_cap, D // 2) == rope_sin.shape
+    q = np.empty((B, Hq, q_cap, D), np.float32)
+    k = np.empty((B, Hkv, q_cap, D), np.float32)
+    v = np.empty((B, Hkv, q_cap, D), np.float32)
+    rc = _load().oracle_qkv_project_rope(B, q_cap, d_model, Hq, Hkv, D, _p(x, np.float32), _p(w, np.float32),
+                                         _p(bias, np.float32), _p(rope_cos, np.float32), _p(rope_sin, np.float32),
+                                         _p(q, np.float32), _p(k, np.float32), _p(v, np.float32))
+    assert rc == 0, rc
+    return q, k, v
+
+
 def out_project(o, wo, bias):
     """o fp32 [B,Hq,q_cap,D], wo fp32 [d_model, Hq*D], bias fp32 [d_model] or None.  Returns y fp32 [B,q_cap,d_model]."""
     B, Hq, q_cap, D = o.shape

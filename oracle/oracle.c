@@ -519,6 +519,59 @@ int oracle_qkv_project(int B, int q_cap, int d_model, int Hq, int Hkv, int D, co
 }
 
 /*
+ * The same projection followed by the rotary position embedding of the query and key heads.  The paper does not
+ * describe the models' position encoding (it runs stock Dream-7B and LLaDA-8B checkpoints, Sec. 4); both use the
+ * rotary embedding of Su et al. (RoFormer) in the half-split layout of their public implementations.  READING taken:
+ * within a head of D features, feature d < D/2 is paired with feature d + D/2, and for the row's angle table
+ * (cos, sin fp32 [B][q_cap][D/2], supplied by the caller for the rows' positions):
+ *     out[d]       = y[d] * cos[d] - y[d + D/2] * sin[d]
+ *     out[d + D/2] = y[d + D/2] * cos[d] + y[d] * sin[d]            (d < D/2; y includes the bias)
+ * applied to the Hq query heads and the Hkv key heads; the value heads are left as they are.  The rotation runs on
+ * the fp64 sums, one rounding to fp32 at the end.
+ */
+int oracle_qkv_project_rope(int B, int q_cap, int d_model, int Hq, int Hkv, int D, const float* x, const float* w,
+                            const float* bias, const float* rope_cos, const float* rope_sin, float* q_out, float* k_out,
+                            float* v_out) {
+  if (D % 2 != 0 || D > 1024) return -1;   /* not a head size this checker handles */
+  const int half = D / 2;
+  const int n_heads = Hq + 2 * Hkv;
+#pragma omp parallel for collapse(2) schedule(static)
+  for (int b = 0; b < B; ++b) {
+    for (int head = 0; head < n_heads; ++head) {
+      float* dst;
+      int heads, h;
+      if (head < Hq) { dst = q_out; heads = Hq; h = head; }
+      else if (head < Hq + Hkv) { dst = k_out; heads = Hkv; h = head - Hq; }
+      else { dst = v_out; heads = Hkv; h = head - Hq - Hkv; }
+      const int rotate = head < Hq + Hkv;
+      double y[1024];
+      for (int i = 0; i < q_cap; ++i) {
+        const float* xr = x + ((size_t)b * q_cap + i) * d_model;
+        for (int d = 0; d < D; ++d) {
+          const int n = head * D + d;
+          const float* wr = w + (size_t)n * d_model;
+          double acc = bias ? (double)bias[n] : 0.0;
+          for (int c = 0; c < d_model; ++c) acc += (double)xr[c] * (double)wr[c];
+          y[d] = acc;
+        }
+        float* out = dst + (((size_t)b * heads + h) * q_cap + i) * D;
+        if (rotate) {
+          const float* cs = rope_cos + ((size_t)b * q_cap + i) * half;
+          const float* sn = rope_sin + ((size_t)b * q_cap + i) * half;
+          for (int d = 0; d < half; ++d) {
+            out[d] = (float)(y[d] * (double)cs[d] - y[d + half] * (double)sn[d]);
+            out[d + half] = (float)(y[d + half] * (double)cs[d] + y[d] * (double)sn[d]);
+          }
+        } else {
+          for (int d = 0; d < D; ++d) out[d] = (float)y[d];
+        }
+      }
+    }
+  }
+  return ORACLE_OK;
+}
+
+/*
  * Output projection (Table 1 row "output projection"): the attention output [B][Hq][q_cap][D], read with features
  * ordered (head, d), times wo [d_model][Hq * D]:
  *     y[b][i][m] = bias[m] + sum_{h,d} o[b][h][i][d] * wo[m][h * D + d]       -> y [B][q_cap][d_model]
