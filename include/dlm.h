@@ -374,6 +374,27 @@ int dlm_window_out_project(dlm_ctx* ctx, const void* o, const void* wo, const vo
                            int d_model, int n_q_heads, int head_dim, void* y, void* workspace,
                            size_t workspace_bytes, void* stream);
 
+/*
+ * dlm_window_qkv_project_rope — dlm_window_qkv_project with the rotary position embedding of the query and key heads
+ * applied in the projection's epilogue, before the one rounding to bf16, so that no separate pass over Q and K sits
+ * between the projection and dlm_freecache_attn_step.  The paper does not describe the models' position encoding (it
+ * runs stock Dream-7B and LLaDA-8B, Sec. 4); both use the rotary embedding of Su et al. (RoFormer) in the half-split
+ * layout.  READING taken (the oracle states the same): within a head, feature d < head_dim / 2 is paired with feature
+ * d + head_dim / 2 and, with the row's angles,
+ *     out[d]                = y[d] * cos[d] - y[d + head_dim / 2] * sin[d]
+ *     out[d + head_dim / 2] = y[d + head_dim / 2] * cos[d] + y[d] * sin[d]          (y includes the bias; fp32)
+ * for the query heads and the key heads; the value heads are written as they are.
+ *   rope_cos, rope_sin   device, fp32 [batch][q_cap][head_dim / 2], 16-byte aligned: cosine and sine of the angle of
+ *                        every (row, pair); the caller computes them from the rows' positions (a window row of
+ *                        sequence b at position t has angle t * base^(-2 d / head_dim) in the usual parametrisation)
+ *   other arguments, workspace and supported shapes as dlm_window_qkv_project; in addition head_dim in {64, 128}
+ *   (DLM_ERR_UNSUPPORTED otherwise), rope_cos and rope_sin not NULL (DLM_ERR_NULL).
+ */
+int dlm_window_qkv_project_rope(dlm_ctx* ctx, const void* x, const void* w, const void* bias, const float* rope_cos,
+                                const float* rope_sin, int batch, int q_cap, int d_model, int n_q_heads,
+                                int n_kv_heads, int head_dim, void* q_out, void* k_out, void* v_out, void* workspace,
+                                size_t workspace_bytes, void* stream);
+
 #ifdef __cplusplus
 }
 #endif

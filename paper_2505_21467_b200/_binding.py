@@ -81,8 +81,10 @@ def lib() -> ctypes.CDLL:
     L.dlm_window_proj_workspace_bytes.argtypes = [vp, i32, i32, i32]
     L.dlm_window_proj_workspace_bytes.restype = sz
     L.dlm_window_qkv_project.argtypes = [vp, vp, vp, vp, i32, i32, i32, i32, i32, i32, vp, vp, vp, vp, sz, vp]
+    L.dlm_window_qkv_project_rope.argtypes = [vp, vp, vp, vp, vp, vp, i32, i32, i32, i32, i32, i32, vp, vp, vp, vp, sz, vp]
     L.dlm_window_out_project.argtypes = [vp, vp, vp, vp, i32, i32, i32, i32, i32, vp, vp, sz, vp]
-    for name in ("dlm_unmask_select_scored", "dlm_guided_accept_threshold", "dlm_window_qkv_project", "dlm_window_out_project"):
+    for name in ("dlm_unmask_select_scored", "dlm_guided_accept_threshold", "dlm_window_qkv_project", "dlm_window_qkv_project_rope",
+                 "dlm_window_out_project"):
         getattr(L, name).restype = i32
     for name in ("dlm_create", "dlm_destroy", "dlm_get_status", "dlm_kv_cache_commit",
                  "dlm_freecache_attn_step", "dlm_unmask_select", "dlm_unmask_select_static", "dlm_guided_accept", "dlm_guided_accept_topk"):
@@ -250,6 +252,15 @@ def dlm_window_qkv_project(ctx, x, w, bias, batch, q_cap, d_model, n_q_heads, n_
         int(n_q_heads), int(n_kv_heads), int(head_dim), _ptr(q_out, torch.bfloat16), _ptr(k_out, torch.bfloat16),
         _ptr(v_out, torch.bfloat16), _ptr(workspace), workspace.numel() * workspace.element_size(), _stream()),
         "dlm_window_qkv_project")
+
+
+def dlm_window_qkv_project_rope(ctx, x, w, bias, rope_cos, rope_sin, batch, q_cap, d_model, n_q_heads, n_kv_heads, head_dim,
+                                q_out, k_out, v_out, workspace) -> None:
+    _check(lib().dlm_window_qkv_project_rope(
+        ctx, _ptr(x, torch.bfloat16), _ptr(w, torch.bfloat16), _ptr(bias, torch.bfloat16), _ptr(rope_cos, torch.float32),
+        _ptr(rope_sin, torch.float32), int(batch), int(q_cap), int(d_model), int(n_q_heads), int(n_kv_heads), int(head_dim),
+        _ptr(q_out, torch.bfloat16), _ptr(k_out, torch.bfloat16), _ptr(v_out, torch.bfloat16), _ptr(workspace),
+        workspace.numel() * workspace.element_size(), _stream()), "dlm_window_qkv_project_rope")
 
 
 def dlm_window_out_project(ctx, o, wo, bias, batch, q_cap, d_model, n_q_heads, head_dim, y, workspace) -> None:

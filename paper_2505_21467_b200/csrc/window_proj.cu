@@ -38,6 +38,8 @@ struct ProjParams {
   __nv_bfloat16* k_out;
   __nv_bfloat16* v_out;
   const __nv_bfloat16* bias;   // [n_out] or nullptr
+  const float* rope_cos;       // mode 0: rotary embedding of the query and key heads, fp32 [B][q_cap][head_dim / 2],
+  const float* rope_sin;       // or both nullptr
   float* partial;              // [row chunk][feature tile][split][rows_pad][128] fp32
   unsigned int* tickets;       // one per (row chunk, feature tile)
   int rows_total, q_cap, n_q_heads, n_kv_heads, head_dim, n_out, k_total;
@@ -65,6 +67,7 @@ window_proj_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_consta
   volatile int* const never_ptr = flags + 1;
   uint32_t* const tmem_slot = reinterpret_cast<uint32_t*>(flags + 2);
   volatile int* const is_last = flags + 3;
+  volatile int* const warp_ok = flags + 4;   // [4]: the epilogue warps' waits, so that all four take the same branches
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int tile = blockIdx.x, split = blockIdx.y, chunk = blockIdx.z;
@@ -164,6 +167,9 @@ window_proj_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_consta
     const int n = tile * kTileN + f;                      // output feature
     bool ok = __all_sync(0xffffffffu, mbar_wait(bar_done, 0, abort_ptr)) != 0;
     tc_fence_after_sync();
+    // rotary embedding (mode 0): feature d of a query or key head is paired with feature d +- head_dim / 2
+    const bool rope = p.mode == 0 && p.rope_cos != nullptr;
+    const int half = p.head_dim >> 1;
     const int rows_here = min(kMaxRows, p.rows_total - row0);
     const size_t tile_slot = ((size_t)chunk * gridDim.x + tile) * p.n_split;
     float* my_partial = p.partial + (tile_slot + split) * (size_t)p.rows_pad * kTileN + f;
@@ -179,7 +185,9 @@ window_proj_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_consta
       }
       __threadfence();
     }
+    if (lane == 0) warp_ok[warp - 2] = ok ? 1 : 0;
     named_bar_sync(1, 128);
+    ok = warp_ok[0] && warp_ok[1] && warp_ok[2] && warp_ok[3];
     if (p.n_split > 1) {
       if (tid == 64) {   // first epilogue thread: every partial store above happened before the barrier
         unsigned int t;
@@ -213,17 +221,35 @@ window_proj_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_consta
       size_t row_stride, b_stride;
       place(n, dst, row_stride, b_stride);
       uint32_t v[32];
+      const bool turn = rope && n / p.head_dim < p.n_q_heads + p.n_kv_heads;   // the same for a feature and its partner
+      const int d = n % p.head_dim;
+      // the partner's values come through shared memory (the pipeline's first stage is free: every MMA has finished);
+      // [feature][33 floats]: 128 x 33 x 4 bytes fit a stage
+      float* const xch = reinterpret_cast<float*>(smem_raw + pad);
+      const int f_partner = d < half ? f + half : f - half;
       for (int c = 0; c < p.rows_pad; c += 32) {
         tmem_ld32(tmem + ((uint32_t)lane_base << 16) + c, v);
         tmem_ld_wait();
+        if (rope) {   // block-uniform: all four warps meet at the two barriers
+#pragma unroll
+          for (int j = 0; j < 32; ++j) xch[f * 33 + j] = __uint_as_float(v[j]) + bias;
+          named_bar_sync(1, 128);
+        }
 #pragma unroll
         for (int j = 0; j < 32; ++j) {
           const int r = row0 + c + j;
           if (c + j < rows_here) {
             const int b = r / p.q_cap, i = r % p.q_cap;
-            dst[(size_t)b * b_stride + (size_t)i * row_stride] = __float2bfloat16_rn(__uint_as_float(v[j]) + bias);
+            float y = __uint_as_float(v[j]) + bias;
+            if (turn) {
+              const size_t a = ((size_t)b * p.q_cap + i) * half + (d < half ? d : d - half);
+              const float cs = p.rope_cos[a], sn = p.rope_sin[a], other = xch[f_partner * 33 + j];
+              y = d < half ? y * cs - other * sn : y * cs + other * sn;
+            }
+            dst[(size_t)b * b_stride + (size_t)i * row_stride] = __float2bfloat16_rn(y);
           }
         }
+        if (rope) named_bar_sync(1, 128);   // the next chunk overwrites the exchange area
       }
     } else if (ok && *is_last) {
       // the last block of the tile adds the partial tiles in split order (the sum does not depend on which block
@@ -250,6 +276,24 @@ window_proj_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_consta
         }
         const int r = row0 + rr;
         const int b = r / p.q_cap, i = r % p.q_cap;
+        if (rope) {
+          // this lane's 4 features and their partners' (head_dim / 2 features = head_dim / 8 lanes away) turn together;
+          // rr is the same for the whole warp, so every lane is here for the exchange
+          const int dl = p.head_dim >> 3;
+          const float4 o = make_float4(__shfl_xor_sync(0xffffffffu, acc.x, dl), __shfl_xor_sync(0xffffffffu, acc.y, dl),
+                                       __shfl_xor_sync(0xffffffffu, acc.z, dl), __shfl_xor_sync(0xffffffffu, acc.w, dl));
+          const int d = n4 % p.head_dim;
+          if (n4 / p.head_dim < p.n_q_heads + p.n_kv_heads) {
+            const size_t a = ((size_t)b * p.q_cap + i) * half + (d < half ? d : d - half);
+            const float4 cs = __ldg(reinterpret_cast<const float4*>(p.rope_cos + a));
+            const float4 sn = __ldg(reinterpret_cast<const float4*>(p.rope_sin + a));
+            const float sg = d < half ? -1.f : 1.f;
+            acc.x = fmaf(sg * o.x, sn.x, acc.x * cs.x);
+            acc.y = fmaf(sg * o.y, sn.y, acc.y * cs.y);
+            acc.z = fmaf(sg * o.z, sn.z, acc.z * cs.z);
+            acc.w = fmaf(sg * o.w, sn.w, acc.w * cs.w);
+          }
+        }
         const __nv_bfloat162 lo = __floats2bfloat162_rn(acc.x, acc.y), hi = __floats2bfloat162_rn(acc.z, acc.w);
         uint2 pk;
         pk.x = *reinterpret_cast<const uint32_t*>(&lo);
@@ -354,9 +398,35 @@ extern "C" size_t dlm_window_proj_workspace_bytes(const dlm_ctx* ctx, int rows, 
   return pl.ws_bytes + 256;
 }
 
+namespace {
+int qkv_project(dlm_ctx* ctx, const void* x, const void* w, const void* bias, const float* rope_cos, const float* rope_sin,
+                int batch, int q_cap, int d_model, int n_q_heads, int n_kv_heads, int head_dim, void* q_out, void* k_out,
+                void* v_out, void* workspace, size_t workspace_bytes, void* stream);
+}
+
 extern "C" int dlm_window_qkv_project(dlm_ctx* ctx, const void* x, const void* w, const void* bias, int batch, int q_cap,
                                       int d_model, int n_q_heads, int n_kv_heads, int head_dim, void* q_out, void* k_out,
                                       void* v_out, void* workspace, size_t workspace_bytes, void* stream) {
+  return qkv_project(ctx, x, w, bias, nullptr, nullptr, batch, q_cap, d_model, n_q_heads, n_kv_heads, head_dim, q_out, k_out,
+                     v_out, workspace, workspace_bytes, stream);
+}
+
+extern "C" int dlm_window_qkv_project_rope(dlm_ctx* ctx, const void* x, const void* w, const void* bias, const float* rope_cos,
+                                           const float* rope_sin, int batch, int q_cap, int d_model, int n_q_heads,
+                                           int n_kv_heads, int head_dim, void* q_out, void* k_out, void* v_out, void* workspace,
+                                           size_t workspace_bytes, void* stream) {
+  if (!rope_cos || !rope_sin) return DLM_ERR_NULL;
+  // a feature and its partner must lie in one 128-feature tile, and 4 neighbouring features in one half of a head
+  if (head_dim != 64 && head_dim != 128) return DLM_ERR_UNSUPPORTED;
+  if (((uintptr_t)rope_cos | (uintptr_t)rope_sin) & 15) return DLM_ERR_UNSUPPORTED;
+  return qkv_project(ctx, x, w, bias, rope_cos, rope_sin, batch, q_cap, d_model, n_q_heads, n_kv_heads, head_dim, q_out, k_out,
+                     v_out, workspace, workspace_bytes, stream);
+}
+
+namespace {
+int qkv_project(dlm_ctx* ctx, const void* x, const void* w, const void* bias, const float* rope_cos, const float* rope_sin,
+                int batch, int q_cap, int d_model, int n_q_heads, int n_kv_heads, int head_dim, void* q_out, void* k_out,
+                void* v_out, void* workspace, size_t workspace_bytes, void* stream) {
   if (!ctx || !x || !w || !q_out || !k_out || !v_out) return DLM_ERR_NULL;
   if (batch <= 0 || q_cap <= 0 || d_model <= 0 || n_q_heads <= 0 || n_kv_heads <= 0 || head_dim <= 0) return DLM_ERR_SHAPE;
   const long long n_out = (long long)(n_q_heads + 2 * n_kv_heads) * head_dim;
@@ -377,10 +447,13 @@ extern "C" int dlm_window_qkv_project(dlm_ctx* ctx, const void* x, const void* w
   p.k_out = static_cast<__nv_bfloat16*>(k_out);
   p.v_out = static_cast<__nv_bfloat16*>(v_out);
   p.bias = static_cast<const __nv_bfloat16*>(bias);
+  p.rope_cos = rope_cos;
+  p.rope_sin = rope_sin;
   p.rows_total = (int)rows; p.q_cap = q_cap; p.n_q_heads = n_q_heads; p.n_kv_heads = n_kv_heads; p.head_dim = head_dim;
   p.n_out = (int)n_out; p.k_total = d_model; p.batch = batch; p.act_heads = 0;
   return launch_proj(ctx, pl, p, tm_w, tm_x, workspace, workspace_bytes, static_cast<cudaStream_t>(stream));
 }
+}  // namespace
 
 extern "C" int dlm_window_out_project(dlm_ctx* ctx, const void* o, const void* wo, const void* bias, int batch, int q_cap,
                                       int d_model, int n_q_heads, int head_dim, void* y, void* workspace,

@@ -102,3 +102,61 @@ def test_projection_argument_errors(dev):
         dlm.dlm_window_out_project(dev.ctx, x, x, None, 2, 13, 128, 2, 128, x, ws)     # batch > 1 needs q_cap % 8 == 0
     assert e.value.code == dlm.DLM_ERR_UNSUPPORTED
     assert dev.status() == 0
+
+
+def _rope_tables(B, q_cap, D, seed, positions=None):
+    """cos / sin fp32 [B][q_cap][D/2]: angles position * base^(-2 d / D), the rows' positions drawn at random."""
+    rng = np.random.default_rng(seed)
+    pos = rng.integers(0, 4096, (B, q_cap)) if positions is None else positions
+    inv = 10000.0 ** (-np.arange(D // 2) * 2.0 / D)
+    th = pos[..., None] * inv
+    return torch.from_numpy(np.cos(th).astype(np.float32)).cuda(), torch.from_numpy(np.sin(th).astype(np.float32)).cuda()
+
+
+@pytest.mark.parametrize("B,q_cap,dm,Hq,Hkv,D,with_bias", [
+    (1, 32, 3584, 28, 4, 128, True),      # Dream-7B widths: K split, the partner feature is 16 lanes away in the final reduction
+    (8, 32, 3584, 28, 4, 128, False),     # 256 rows
+    (4, 64, 4096, 32, 32, 128, False),    # LLaDA-8B widths
+    (1, 20, 512, 4, 2, 128, True),        # ragged rows
+    (3, 100, 256, 2, 1, 128, True),       # two row chunks
+    (2, 7, 128, 4, 2, 64, False),         # head_dim 64, K too short to split: the partner comes through shared memory
+    (2, 40, 1024, 6, 3, 64, True),        # head_dim 64 with the K split: two heads per tile, partner 8 lanes away; a tile
+                                          # straddles the last key head and the first value head
+    (1, 9, 128, 1, 1, 128, True),         # K too short to split, head_dim 128: the partner sits in another warp
+])
+def test_qkv_projection_with_rotary_embedding(dev, oracle, B, q_cap, dm, Hq, Hkv, D, with_bias):
+    seed = 7 * B + q_cap
+    n_out = (Hq + 2 * Hkv) * D
+    x = make_kv_rows((B, q_cap, dm), seed, "cuda")
+    w = (torch.randn(n_out, dm, generator=torch.Generator("cuda").manual_seed(seed + 1), device="cuda") * dm ** -0.5).to(torch.bfloat16)
+    bias = make_kv_rows((n_out,), seed + 2, "cuda") if with_bias else None
+    cs, sn = _rope_tables(B, q_cap, D, seed + 3)
+    nan = float("nan")
+    q = torch.full((B, Hq, q_cap, D), nan, dtype=torch.bfloat16, device="cuda")
+    k = torch.full((B, Hkv, q_cap, D), nan, dtype=torch.bfloat16, device="cuda")
+    v = torch.full((B, Hkv, q_cap, D), nan, dtype=torch.bfloat16, device="cuda")
+    ws = dev.workspace(dlm.dlm_window_proj_workspace_bytes(dev.ctx, B * q_cap, n_out, dm))
+    dlm.dlm_window_qkv_project_rope(dev.ctx, x, w, bias, cs, sn, B, q_cap, dm, Hq, Hkv, D, q, k, v, ws)
+    assert dev.status() == 0
+    rq, rk, rv = oracle.qkv_project_rope(widen(x), widen(w), None if bias is None else widen(bias), cs.cpu().numpy(),
+                                         sn.cpu().numpy(), Hq, Hkv, D)
+    _close(q, rq, "q"); _close(k, rk, "k"); _close(v, rv, "v")
+    # the value heads are exactly those of the plain call
+    q2, k2, v2 = torch.empty_like(q), torch.empty_like(k), torch.empty_like(v)
+    dlm.dlm_window_qkv_project(dev.ctx, x, w, bias, B, q_cap, dm, Hq, Hkv, D, q2, k2, v2, ws)
+    assert torch.equal(v, v2) and not torch.equal(q, q2)
+
+
+def test_rotary_projection_argument_errors(dev):
+    x = torch.zeros(1, 8, 64, dtype=torch.bfloat16, device="cuda")
+    w = torch.zeros(3 * 32 * 4, 64, dtype=torch.bfloat16, device="cuda")
+    t = torch.zeros(1, 8, 16, device="cuda")
+    o = torch.zeros(1, 4, 8, 32, dtype=torch.bfloat16, device="cuda")
+    ws = dev.workspace(1 << 20)
+    with pytest.raises(dlm.DlmError) as e:     # head_dim 32
+        dlm.dlm_window_qkv_project_rope(dev.ctx, x, w, None, t, t, 1, 8, 64, 4, 4, 32, o, o, o, ws)
+    assert e.value.code == dlm.DLM_ERR_UNSUPPORTED
+    with pytest.raises(dlm.DlmError) as e:
+        dlm.dlm_window_qkv_project_rope(dev.ctx, x, w, None, None, t, 1, 8, 64, 4, 4, 32, o, o, o, ws)
+    assert e.value.code == dlm.DLM_ERR_NULL
+    assert dev.status() == 0
