@@ -395,6 +395,29 @@ int dlm_window_qkv_project_rope(dlm_ctx* ctx, const void* x, const void* w, cons
                                 int n_kv_heads, int head_dim, void* q_out, void* k_out, void* v_out, void* workspace,
                                 size_t workspace_bytes, void* stream);
 
+/*
+ * dlm_window_qkv_project_stage — the projection (with the rotary embedding when rope_cos / rope_sin are given, as
+ * dlm_window_qkv_project_rope; both NULL: none) that also stages the window's K/V rows in the cache from its epilogue
+ * (Sec. 3.2.1 "Windowed Re-computation": the active block's K/V are recomputed in every step; "upon completion of
+ * block B_i, its KV projections are frozen").  Beside k_out / v_out, row i of sequence b is written to cache row
+ * cache_len[b] + i of layer `layer` (K and V), the slot dlm_kv_cache_commit's DLM_DST_WINDOW mode uses, with the
+ * same bits as in k_out / v_out.  cache_len is not changed: the staged rows stay invisible to
+ * dlm_freecache_attn_step until the caller advances cache_len[b] by the block's length when the block is complete,
+ * and the rows staged by the block's last step are then the frozen ones; no separate copy of the block is needed.
+ *   q_len   device, int32 [batch] or NULL: only rows i < q_len[b] are staged (NULL: all q_cap rows); q_out, k_out
+ *           and v_out hold all q_cap rows either way
+ *   cache   its k / v / cache_len are device pointers as for dlm_kv_cache_commit; batch, n_kv_heads and head_dim
+ *           must match the call's (DLM_ERR_SHAPE), 0 <= layer < n_layers
+ * Data-dependent: a row whose slot lies at or beyond the capacity is not staged and DLM_ERR_CAPACITY is recorded.
+ * A step of a model then needs no dlm_kv_cache_commit call at all; the commit entry point remains for refreshes
+ * and for rows chosen after the fact.
+ */
+int dlm_window_qkv_project_stage(dlm_ctx* ctx, const void* x, const void* w, const void* bias, const float* rope_cos,
+                                 const float* rope_sin, int batch, int q_cap, int d_model, int n_q_heads,
+                                 int n_kv_heads, int head_dim, const int32_t* q_len, void* q_out, void* k_out,
+                                 void* v_out, const dlm_kv_cache* cache, int layer, void* workspace,
+                                 size_t workspace_bytes, void* stream);
+
 #ifdef __cplusplus
 }
 #endif

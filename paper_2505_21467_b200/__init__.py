@@ -11,6 +11,6 @@ from ._binding import (  # noqa: F401
     dlm_kv_cache_commit, dlm_attn_workspace_bytes, dlm_freecache_attn_step,
     dlm_unmask_workspace_bytes, dlm_unmask_select, dlm_unmask_select_static, dlm_guided_accept, dlm_guided_accept_topk,
     dlm_unmask_scored_workspace_bytes, dlm_unmask_select_scored, dlm_guided_accept_threshold,
-    dlm_window_proj_workspace_bytes, dlm_window_qkv_project, dlm_window_qkv_project_rope, dlm_window_out_project,
+    dlm_window_proj_workspace_bytes, dlm_window_qkv_project, dlm_window_qkv_project_rope, dlm_window_qkv_project_stage, dlm_window_out_project,
     DLM_SCORE_CONFIDENCE, DLM_SCORE_NEG_ENTROPY, DLM_SCORE_MARGIN, DLM_SCORE_LOG_CONF_PLUS_NOISE,
 )

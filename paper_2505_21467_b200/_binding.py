@@ -82,6 +82,9 @@ def lib() -> ctypes.CDLL:
     L.dlm_window_proj_workspace_bytes.restype = sz
     L.dlm_window_qkv_project.argtypes = [vp, vp, vp, vp, i32, i32, i32, i32, i32, i32, vp, vp, vp, vp, sz, vp]
     L.dlm_window_qkv_project_rope.argtypes = [vp, vp, vp, vp, vp, vp, i32, i32, i32, i32, i32, i32, vp, vp, vp, vp, sz, vp]
+    L.dlm_window_qkv_project_stage.argtypes = [vp, vp, vp, vp, vp, vp, i32, i32, i32, i32, i32, i32, vp, vp, vp, vp,
+                                               ctypes.POINTER(dlm_kv_cache), i32, vp, sz, vp]
+    L.dlm_window_qkv_project_stage.restype = i32
     L.dlm_window_out_project.argtypes = [vp, vp, vp, vp, i32, i32, i32, i32, i32, vp, vp, sz, vp]
     for name in ("dlm_unmask_select_scored", "dlm_guided_accept_threshold", "dlm_window_qkv_project", "dlm_window_qkv_project_rope",
                  "dlm_window_out_project"):
@@ -261,6 +264,16 @@ def dlm_window_qkv_project_rope(ctx, x, w, bias, rope_cos, rope_sin, batch, q_ca
         _ptr(rope_sin, torch.float32), int(batch), int(q_cap), int(d_model), int(n_q_heads), int(n_kv_heads), int(head_dim),
         _ptr(q_out, torch.bfloat16), _ptr(k_out, torch.bfloat16), _ptr(v_out, torch.bfloat16), _ptr(workspace),
         workspace.numel() * workspace.element_size(), _stream()), "dlm_window_qkv_project_rope")
+
+
+def dlm_window_qkv_project_stage(ctx, x, w, bias, rope_cos, rope_sin, batch, q_cap, d_model, n_q_heads, n_kv_heads, head_dim,
+                                 q_len, q_out, k_out, v_out, cache, layer, workspace) -> None:
+    _check(lib().dlm_window_qkv_project_stage(
+        ctx, _ptr(x, torch.bfloat16), _ptr(w, torch.bfloat16), _ptr(bias, torch.bfloat16), _ptr(rope_cos, torch.float32),
+        _ptr(rope_sin, torch.float32), int(batch), int(q_cap), int(d_model), int(n_q_heads), int(n_kv_heads), int(head_dim),
+        _ptr(q_len, torch.int32), _ptr(q_out, torch.bfloat16), _ptr(k_out, torch.bfloat16), _ptr(v_out, torch.bfloat16),
+        ctypes.byref(cache), int(layer), _ptr(workspace), workspace.numel() * workspace.element_size(), _stream()),
+        "dlm_window_qkv_project_stage")
 
 
 def dlm_window_out_project(ctx, o, wo, bias, batch, q_cap, d_model, n_q_heads, head_dim, y, workspace) -> None:

@@ -40,6 +40,13 @@ struct ProjParams {
   const __nv_bfloat16* bias;   // [n_out] or nullptr
   const float* rope_cos;       // mode 0: rotary embedding of the query and key heads, fp32 [B][q_cap][head_dim / 2],
   const float* rope_sin;       // or both nullptr
+  // mode 0: K/V rows are also staged in the cache (one layer: [B][n_kv_heads][capacity][head_dim]) at row
+  // cache_len[b] + i, the slot the commit's window mode uses; nullptr: no staging
+  __nv_bfloat16* stage_k;
+  __nv_bfloat16* stage_v;
+  const int32_t* cache_len;    // [B]
+  const int32_t* q_len;        // [B] rows of the window that are active (staged), or nullptr: all q_cap
+  int capacity;
   float* partial;              // [row chunk][feature tile][split][rows_pad][128] fp32
   unsigned int* tickets;       // one per (row chunk, feature tile)
   int rows_total, q_cap, n_q_heads, n_kv_heads, head_dim, n_out, k_total;
@@ -198,14 +205,18 @@ window_proj_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_consta
       named_bar_sync(1, 128);
     }
     // where output feature `feat` of row (b, i) goes: element offset of (b = 0, i = 0) and the two strides
-    auto place = [&](int feat, __nv_bfloat16*& dst, size_t& row_stride, size_t& b_stride) {
+    // ... and, for a key or value feature of a staging call, where its copy in the cache goes: element offset of
+    // (b = 0, cache row 0); rows are head_dim apart, batch elements n_kv_heads * capacity * head_dim
+    auto place = [&](int feat, __nv_bfloat16*& dst, size_t& row_stride, size_t& b_stride, __nv_bfloat16*& stage) {
+      stage = nullptr;
       if (p.mode == 0) {
         const int head = feat / p.head_dim, d = feat % p.head_dim;
         int heads, h;
         if (head < p.n_q_heads) { dst = p.q_out; heads = p.n_q_heads; h = head; }
-        else if (head < p.n_q_heads + p.n_kv_heads) { dst = p.k_out; heads = p.n_kv_heads; h = head - p.n_q_heads; }
-        else { dst = p.v_out; heads = p.n_kv_heads; h = head - p.n_q_heads - p.n_kv_heads; }
+        else if (head < p.n_q_heads + p.n_kv_heads) { dst = p.k_out; heads = p.n_kv_heads; h = head - p.n_q_heads; stage = p.stage_k; }
+        else { dst = p.v_out; heads = p.n_kv_heads; h = head - p.n_q_heads - p.n_kv_heads; stage = p.stage_v; }
         dst += (size_t)h * p.q_cap * p.head_dim + d;
+        if (stage) stage += (size_t)h * p.capacity * p.head_dim + d;
         row_stride = p.head_dim;
         b_stride = (size_t)heads * p.q_cap * p.head_dim;
       } else {
@@ -214,12 +225,24 @@ window_proj_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_consta
         b_stride = (size_t)p.q_cap * p.n_out;
       }
     };
+    // cache row that window row i of batch element b is staged at, or -1: inactive row, or no room (reported)
+    auto stage_row = [&](int b, int i) -> int {
+      if (p.q_len && i >= __ldg(p.q_len + b)) return -1;
+      const int pos = __ldg(p.cache_len + b) + i;
+      if (pos < 0 || pos >= p.capacity) {
+        dlm_set_status(p.status, DLM_ERR_CAPACITY);
+        return -1;
+      }
+      return pos;
+    };
+    const size_t stage_b_stride = (size_t)p.n_kv_heads * p.capacity * p.head_dim;
     if (ok && p.n_split == 1) {
       // the whole sum is in TMEM: thread = feature, one 2-byte store per row (the output is small beside the weights)
       const float bias = p.bias ? __bfloat162float(p.bias[n]) : 0.f;
       __nv_bfloat16* dst;
+      __nv_bfloat16* stage;
       size_t row_stride, b_stride;
-      place(n, dst, row_stride, b_stride);
+      place(n, dst, row_stride, b_stride, stage);
       uint32_t v[32];
       const bool turn = rope && n / p.head_dim < p.n_q_heads + p.n_kv_heads;   // the same for a feature and its partner
       const int d = n % p.head_dim;
@@ -246,7 +269,12 @@ window_proj_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_consta
               const float cs = p.rope_cos[a], sn = p.rope_sin[a], other = xch[f_partner * 33 + j];
               y = d < half ? y * cs - other * sn : y * cs + other * sn;
             }
-            dst[(size_t)b * b_stride + (size_t)i * row_stride] = __float2bfloat16_rn(y);
+            const __nv_bfloat16 yb = __float2bfloat16_rn(y);
+            dst[(size_t)b * b_stride + (size_t)i * row_stride] = yb;
+            if (stage) {
+              const int pos = stage_row(b, i);
+              if (pos >= 0) stage[(size_t)b * stage_b_stride + (size_t)pos * p.head_dim] = yb;
+            }
           }
         }
         if (rope) named_bar_sync(1, 128);   // the next chunk overwrites the exchange area
@@ -263,8 +291,9 @@ window_proj_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_consta
       if (p.bias)
         for (int j = 0; j < 4; ++j) b4[j] = __bfloat162float(p.bias[n4 + j]);
       __nv_bfloat16* dst;
+      __nv_bfloat16* stage;
       size_t row_stride, b_stride;
-      place(n4, dst, row_stride, b_stride);
+      place(n4, dst, row_stride, b_stride, stage);
       const float* src0 = p.partial + tile_slot * (size_t)p.rows_pad * kTileN + fq;
       const size_t split_stride = (size_t)p.rows_pad * kTileN;
 #pragma unroll 4
@@ -299,6 +328,10 @@ window_proj_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_consta
         pk.x = *reinterpret_cast<const uint32_t*>(&lo);
         pk.y = *reinterpret_cast<const uint32_t*>(&hi);
         *reinterpret_cast<uint2*>(dst + (size_t)b * b_stride + (size_t)i * row_stride) = pk;
+        if (stage) {
+          const int pos = stage_row(b, i);
+          if (pos >= 0) *reinterpret_cast<uint2*>(stage + (size_t)b * stage_b_stride + (size_t)pos * p.head_dim) = pk;
+        }
       }
     }
   }
@@ -401,14 +434,15 @@ extern "C" size_t dlm_window_proj_workspace_bytes(const dlm_ctx* ctx, int rows, 
 namespace {
 int qkv_project(dlm_ctx* ctx, const void* x, const void* w, const void* bias, const float* rope_cos, const float* rope_sin,
                 int batch, int q_cap, int d_model, int n_q_heads, int n_kv_heads, int head_dim, void* q_out, void* k_out,
-                void* v_out, void* workspace, size_t workspace_bytes, void* stream);
+                void* v_out, const dlm_kv_cache* cache, int layer, const int32_t* q_len, void* workspace, size_t workspace_bytes,
+                void* stream);
 }
 
 extern "C" int dlm_window_qkv_project(dlm_ctx* ctx, const void* x, const void* w, const void* bias, int batch, int q_cap,
                                       int d_model, int n_q_heads, int n_kv_heads, int head_dim, void* q_out, void* k_out,
                                       void* v_out, void* workspace, size_t workspace_bytes, void* stream) {
   return qkv_project(ctx, x, w, bias, nullptr, nullptr, batch, q_cap, d_model, n_q_heads, n_kv_heads, head_dim, q_out, k_out,
-                     v_out, workspace, workspace_bytes, stream);
+                     v_out, nullptr, 0, nullptr, workspace, workspace_bytes, stream);
 }
 
 extern "C" int dlm_window_qkv_project_rope(dlm_ctx* ctx, const void* x, const void* w, const void* bias, const float* rope_cos,
@@ -420,13 +454,30 @@ extern "C" int dlm_window_qkv_project_rope(dlm_ctx* ctx, const void* x, const vo
   if (head_dim != 64 && head_dim != 128) return DLM_ERR_UNSUPPORTED;
   if (((uintptr_t)rope_cos | (uintptr_t)rope_sin) & 15) return DLM_ERR_UNSUPPORTED;
   return qkv_project(ctx, x, w, bias, rope_cos, rope_sin, batch, q_cap, d_model, n_q_heads, n_kv_heads, head_dim, q_out, k_out,
-                     v_out, workspace, workspace_bytes, stream);
+                     v_out, nullptr, 0, nullptr, workspace, workspace_bytes, stream);
+}
+
+extern "C" int dlm_window_qkv_project_stage(dlm_ctx* ctx, const void* x, const void* w, const void* bias, const float* rope_cos,
+                                            const float* rope_sin, int batch, int q_cap, int d_model, int n_q_heads,
+                                            int n_kv_heads, int head_dim, const int32_t* q_len, void* q_out, void* k_out,
+                                            void* v_out, const dlm_kv_cache* cache, int layer, void* workspace,
+                                            size_t workspace_bytes, void* stream) {
+  if (!cache || !cache->k || !cache->v || !cache->cache_len) return DLM_ERR_NULL;
+  if ((rope_cos == nullptr) != (rope_sin == nullptr)) return DLM_ERR_NULL;
+  if (rope_cos && head_dim != 64 && head_dim != 128) return DLM_ERR_UNSUPPORTED;
+  if (((uintptr_t)rope_cos | (uintptr_t)rope_sin | (uintptr_t)cache->k | (uintptr_t)cache->v) & 15) return DLM_ERR_UNSUPPORTED;
+  if (layer < 0 || layer >= cache->n_layers || cache->batch != batch || cache->n_kv_heads != n_kv_heads ||
+      cache->head_dim != head_dim || cache->capacity <= 0)
+    return DLM_ERR_SHAPE;
+  return qkv_project(ctx, x, w, bias, rope_cos, rope_sin, batch, q_cap, d_model, n_q_heads, n_kv_heads, head_dim, q_out, k_out,
+                     v_out, cache, layer, q_len, workspace, workspace_bytes, stream);
 }
 
 namespace {
 int qkv_project(dlm_ctx* ctx, const void* x, const void* w, const void* bias, const float* rope_cos, const float* rope_sin,
                 int batch, int q_cap, int d_model, int n_q_heads, int n_kv_heads, int head_dim, void* q_out, void* k_out,
-                void* v_out, void* workspace, size_t workspace_bytes, void* stream) {
+                void* v_out, const dlm_kv_cache* cache, int layer, const int32_t* q_len, void* workspace, size_t workspace_bytes,
+                void* stream) {
   if (!ctx || !x || !w || !q_out || !k_out || !v_out) return DLM_ERR_NULL;
   if (batch <= 0 || q_cap <= 0 || d_model <= 0 || n_q_heads <= 0 || n_kv_heads <= 0 || head_dim <= 0) return DLM_ERR_SHAPE;
   const long long n_out = (long long)(n_q_heads + 2 * n_kv_heads) * head_dim;
@@ -449,6 +500,14 @@ int qkv_project(dlm_ctx* ctx, const void* x, const void* w, const void* bias, co
   p.bias = static_cast<const __nv_bfloat16*>(bias);
   p.rope_cos = rope_cos;
   p.rope_sin = rope_sin;
+  if (cache) {
+    const size_t layer_elems = (size_t)batch * n_kv_heads * cache->capacity * head_dim;
+    p.stage_k = static_cast<__nv_bfloat16*>(cache->k) + (size_t)layer * layer_elems;
+    p.stage_v = static_cast<__nv_bfloat16*>(cache->v) + (size_t)layer * layer_elems;
+    p.cache_len = cache->cache_len;
+    p.q_len = q_len;
+    p.capacity = cache->capacity;
+  }
   p.rows_total = (int)rows; p.q_cap = q_cap; p.n_q_heads = n_q_heads; p.n_kv_heads = n_kv_heads; p.head_dim = head_dim;
   p.n_out = (int)n_out; p.k_total = d_model; p.batch = batch; p.act_heads = 0;
   return launch_proj(ctx, pl, p, tm_w, tm_x, workspace, workspace_bytes, static_cast<cudaStream_t>(stream));
