@@ -250,34 +250,50 @@ window_proj_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_consta
       // [feature][33 floats]: 128 x 33 x 4 bytes fit a stage
       float* const xch = reinterpret_cast<float*>(smem_raw + pad);
       const int f_partner = d < half ? f + half : f - half;
-      for (int c = 0; c < p.rows_pad; c += 32) {
-        tmem_ld32(tmem + ((uint32_t)lane_base << 16) + c, v);
-        tmem_ld_wait();
-        if (rope) {   // block-uniform: all four warps meet at the two barriers
+      if (!rope && !stage) {
+        // the plain projection: nothing but the bias between the accumulator and the store
+        for (int c = 0; c < p.rows_pad; c += 32) {
+          tmem_ld32(tmem + ((uint32_t)lane_base << 16) + c, v);
+          tmem_ld_wait();
 #pragma unroll
-          for (int j = 0; j < 32; ++j) xch[f * 33 + j] = __uint_as_float(v[j]) + bias;
-          named_bar_sync(1, 128);
-        }
-#pragma unroll
-        for (int j = 0; j < 32; ++j) {
-          const int r = row0 + c + j;
-          if (c + j < rows_here) {
-            const int b = r / p.q_cap, i = r % p.q_cap;
-            float y = __uint_as_float(v[j]) + bias;
-            if (turn) {
-              const size_t a = ((size_t)b * p.q_cap + i) * half + (d < half ? d : d - half);
-              const float cs = p.rope_cos[a], sn = p.rope_sin[a], other = xch[f_partner * 33 + j];
-              y = d < half ? y * cs - other * sn : y * cs + other * sn;
-            }
-            const __nv_bfloat16 yb = __float2bfloat16_rn(y);
-            dst[(size_t)b * b_stride + (size_t)i * row_stride] = yb;
-            if (stage) {
-              const int pos = stage_row(b, i);
-              if (pos >= 0) stage[(size_t)b * stage_b_stride + (size_t)pos * p.head_dim] = yb;
+          for (int j = 0; j < 32; ++j) {
+            const int r = row0 + c + j;
+            if (c + j < rows_here) {
+              const int b = r / p.q_cap, i = r % p.q_cap;
+              dst[(size_t)b * b_stride + (size_t)i * row_stride] = __float2bfloat16_rn(__uint_as_float(v[j]) + bias);
             }
           }
         }
-        if (rope) named_bar_sync(1, 128);   // the next chunk overwrites the exchange area
+      } else {
+        for (int c = 0; c < p.rows_pad; c += 32) {
+          tmem_ld32(tmem + ((uint32_t)lane_base << 16) + c, v);
+          tmem_ld_wait();
+          if (rope) {   // block-uniform: all four warps meet at the two barriers
+#pragma unroll
+            for (int j = 0; j < 32; ++j) xch[f * 33 + j] = __uint_as_float(v[j]) + bias;
+            named_bar_sync(1, 128);
+          }
+#pragma unroll
+          for (int j = 0; j < 32; ++j) {
+            const int r = row0 + c + j;
+            if (c + j < rows_here) {
+              const int b = r / p.q_cap, i = r % p.q_cap;
+              float y = __uint_as_float(v[j]) + bias;
+              if (turn) {
+                const size_t a = ((size_t)b * p.q_cap + i) * half + (d < half ? d : d - half);
+                const float cs = p.rope_cos[a], sn = p.rope_sin[a], other = xch[f_partner * 33 + j];
+                y = d < half ? y * cs - other * sn : y * cs + other * sn;
+              }
+              const __nv_bfloat16 yb = __float2bfloat16_rn(y);
+              dst[(size_t)b * b_stride + (size_t)i * row_stride] = yb;
+              if (stage) {
+                const int pos = stage_row(b, i);
+                if (pos >= 0) stage[(size_t)b * stage_b_stride + (size_t)pos * p.head_dim] = yb;
+              }
+            }
+          }
+          if (rope) named_bar_sync(1, 128);   // the next chunk overwrites the exchange area
+        }
       }
     } else if (ok && *is_last) {
       // the last block of the tile adds the partial tiles in split order (the sum does not depend on which block
