@@ -304,6 +304,9 @@ __device__ __noinline__ void team_publish(const TeamArgs p, const int* prefix, u
     *arrive = 0;
     *depart = 0;
   }
+  // the copies issued above land in this block's shared memory: this thread does not leave before they have (the
+  // softmax threads wait on the same barrier, but may have given up); abort_ptr + 1 is the flag that stays 0
+  mbar_wait(bar_team, 0, abort_ptr + 1);
 }
 
 // Softmax threads (all live ones of the block, whole warps): store this thread's row of the block's piece --
