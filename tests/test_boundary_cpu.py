@@ -3,6 +3,8 @@ import ctypes
 import os
 import re
 
+import pytest
+
 ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
 
 
@@ -47,3 +49,17 @@ def test_product_package_never_imports_the_oracle():
             if f.endswith((".py", ".cu", ".cuh", ".h")):
                 src = open(os.path.join(dirpath, f)).read()
                 assert "oracle" not in src, f"{f} mentions the oracle"
+
+
+def test_build_checks_the_attention_kernels_register_count():
+    """The attention kernel's setmaxnreg split balances only at 168 registers per thread at launch: the build reads
+    ptxas's log and refuses any other number (a run-time DLM_ERR_UNSUPPORTED otherwise)."""
+    from paper_2505_21467_b200 import build as b
+    ok = ("ptxas info    : Compiling entry function '_ZN3foo22attn_step_sm100_kernelILi128ELi256ELb0EEEv' for 'sm_100a'\n"
+          "ptxas info    : Used 168 registers, used 1 barriers\n"
+          "ptxas info    : Compiling entry function 'other_kernel' for 'sm_100a'\nptxas info    : Used 40 registers\n")
+    b.check_attention_registers(ok)
+    with pytest.raises(RuntimeError):
+        b.check_attention_registers(ok.replace("Used 168", "Used 160"))
+    with pytest.raises(RuntimeError):
+        b.check_attention_registers("ptxas info    : Compiling entry function 'other_kernel' for 'sm_100a'\nptxas info    : Used 40 registers\n")
