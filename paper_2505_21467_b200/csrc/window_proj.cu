@@ -58,7 +58,22 @@ struct ProjParams {
   int* status;
 };
 
-__device__ __forceinline__ void tmem_ld32_nowait(uint32_t taddr, uint32_t* r) { tmem_ld32(taddr, r); }
+// Waits until the counter at `addr` reaches `target` (acquire, device scope), bounded like the mbarrier waits.
+__device__ __forceinline__ bool wait_count(const unsigned int* addr, unsigned int target, volatile int* abort_flag) {
+  const uint64_t t0 = global_timer_ns();
+  for (uint32_t spin = 1;; ++spin) {
+    unsigned int v;
+    asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(addr) : "memory");
+    if (v >= target) return true;
+    if ((spin & 15u) == 0u) {
+      if (*abort_flag) return false;
+      if (global_timer_ns() - t0 > kWaitLimitNs) {
+        *abort_flag = 1;
+        return false;
+      }
+    }
+  }
+}
 
 __global__ void __launch_bounds__(kThreads, 1)
 window_proj_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ CUtensorMap tm_x, const ProjParams p) {
@@ -69,6 +84,7 @@ window_proj_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_consta
   const uint32_t stage_bytes = kWBytes + x_bytes;
   const uint32_t sm_bar = base + p.n_stages * stage_bytes;          // full[8], empty[8], done
   const uint32_t bar_full = sm_bar, bar_empty = sm_bar + 8 * kMaxStages, bar_done = sm_bar + 16 * kMaxStages;
+  const uint32_t bar_red = bar_done + 8;   // the partial tiles' slices of this block's rows have landed in shared memory
   int* const flags = reinterpret_cast<int*>(smem_raw + pad + (size_t)p.n_stages * stage_bytes + 16 * kMaxStages + 16);
   volatile int* const abort_ptr = flags;
   volatile int* const never_ptr = flags + 1;
@@ -92,6 +108,7 @@ window_proj_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_consta
       mbar_init(bar_empty + 8 * i, 1);
     }
     mbar_init(bar_done, 1);
+    mbar_init(bar_red, 1);
     mbar_fence_init();
     fence_proxy_async_smem();
   }
@@ -195,12 +212,36 @@ window_proj_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_consta
     if (lane == 0) warp_ok[warp - 2] = ok ? 1 : 0;
     named_bar_sync(1, 128);
     ok = warp_ok[0] && warp_ok[1] && warp_ok[2] && warp_ok[3];
+    // Split K: the n_split blocks of a tile share its final reduction.  Block s takes rows [lo, hi) of the tile; when
+    // all partial tiles are there (arrival counter; the blocks of a launch are all resident: there are no more of
+    // them than SMs) it fetches those rows of every partial tile into the shared memory of the pipeline stages, which
+    // are free by now, with bulk copies, all in flight at once.  (One block folding the other partial tiles with
+    // loads of its own took 6 us of a 16 us call at 32 rows and 37 of 52 us at 256: every batch of loads is a trip of
+    // about 2 us to data other SMs have just written.)  A second counter lets the last block to leave clear both.
+    const int red_lo = p.rows_pad * split / p.n_split, red_hi = p.rows_pad * (split + 1) / p.n_split;
+    const uint32_t slice_bytes = (uint32_t)(red_hi - red_lo) * kTileN * 4u;
     if (p.n_split > 1) {
       if (tid == 64) {   // first epilogue thread: every partial store above happened before the barrier
-        unsigned int t;
-        asm volatile("atom.acq_rel.gpu.global.add.u32 %0, [%1], 1;" : "=r"(t) : "l"(p.tickets + chunk * gridDim.x + tile) : "memory");
-        *is_last = (t == (unsigned int)p.n_split - 1u) ? 1 : 0;
-        if (*is_last) p.tickets[chunk * gridDim.x + tile] = 0;
+        int go = 2;
+        unsigned int* const arrive = p.tickets + chunk * gridDim.x + tile;
+        unsigned int* const depart = arrive + kDlmMaxSplitUnits / 2;
+        if (ok) {
+          unsigned int t;
+          asm volatile("atom.acq_rel.gpu.global.add.u32 %0, [%1], 1;" : "=r"(t) : "l"(arrive) : "memory");
+          if (wait_count(arrive, (unsigned int)p.n_split, abort_ptr)) {
+            fence_proxy_async_all();
+            mbar_expect_tx(bar_red, (uint32_t)p.n_split * slice_bytes);
+            for (int s2 = 0; s2 < p.n_split; ++s2)
+              bulk_load(base + s2 * slice_bytes, p.partial + ((tile_slot + s2) * (size_t)p.rows_pad + red_lo) * kTileN, slice_bytes,
+                        bar_red);
+            if (atomicAdd(depart, 1u) == (unsigned int)p.n_split - 1u) {   // every block of the tile is past its wait
+              *arrive = 0;
+              *depart = 0;
+            }
+            go = 1;
+          }
+        }
+        *is_last = go;
       }
       named_bar_sync(1, 128);
     }
@@ -295,11 +336,13 @@ window_proj_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_consta
           if (rope) named_bar_sync(1, 128);   // the next chunk overwrites the exchange area
         }
       }
-    } else if (ok && *is_last) {
-      // the last block of the tile adds the partial tiles in split order (the sum does not depend on which block
-      // came last): a thread takes 4 neighbouring features of every fourth row, 16-byte loads, 8-byte stores; a
+    } else if (ok && *is_last == 1) {
+      // every block adds its rows of the partial tiles in split order (the sum does not depend on the order of arrival): a
+      // thread takes 4 neighbouring features of every fourth row, 16-byte loads from shared memory, 8-byte stores; a
       // warp's stores cover 128 features of one row
-      __threadfence();
+      const bool landed = __all_sync(0xffffffffu, mbar_wait(bar_red, 0, abort_ptr)) != 0;
+      // the thread that issued the copies does not go on to the teardown before they have landed
+      if (tid == 64 && !landed) mbar_wait(bar_red, 0, never_ptr);
       const int t = tid - 64;
       const int fq = (t & 31) * 4;
       const int n4 = tile * kTileN + fq;
@@ -310,43 +353,53 @@ window_proj_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_consta
       __nv_bfloat16* stage;
       size_t row_stride, b_stride;
       place(n4, dst, row_stride, b_stride, stage);
-      const float* src0 = p.partial + tile_slot * (size_t)p.rows_pad * kTileN + fq;
-      const size_t split_stride = (size_t)p.rows_pad * kTileN;
-#pragma unroll 4
-      for (int rr = t >> 5; rr < rows_here; rr += 4) {
-        float4 acc = make_float4(b4[0], b4[1], b4[2], b4[3]);
+      const int red_end = landed ? min(red_hi, rows_here) : red_lo;   // rows beyond the call's hold nothing
+      for (int rr0 = red_lo + (t >> 5); rr0 < red_end; rr0 += 16) {
+        float4 accs[4];
+#pragma unroll
+        for (int j = 0; j < 4; ++j) accs[j] = make_float4(b4[0], b4[1], b4[2], b4[3]);
         for (int s2 = 0; s2 < p.n_split; ++s2) {
-          const float4 x = __ldcg(reinterpret_cast<const float4*>(src0 + s2 * split_stride + (size_t)rr * kTileN));
-          acc.x += x.x; acc.y += x.y; acc.z += x.z; acc.w += x.w;
+#pragma unroll
+          for (int j = 0; j < 4; ++j)
+            if (rr0 + 4 * j < red_end) {
+              const float4 x = ld_shared_f4(base + s2 * slice_bytes + (uint32_t)((rr0 + 4 * j - red_lo) * kTileN + fq) * 4u);
+              accs[j].x += x.x; accs[j].y += x.y; accs[j].z += x.z; accs[j].w += x.w;
+            }
         }
-        const int r = row0 + rr;
-        const int b = r / p.q_cap, i = r % p.q_cap;
-        if (rope) {
-          // this lane's 4 features and their partners' (head_dim / 2 features = head_dim / 8 lanes away) turn together;
-          // rr is the same for the whole warp, so every lane is here for the exchange
-          const int dl = p.head_dim >> 3;
-          const float4 o = make_float4(__shfl_xor_sync(0xffffffffu, acc.x, dl), __shfl_xor_sync(0xffffffffu, acc.y, dl),
-                                       __shfl_xor_sync(0xffffffffu, acc.z, dl), __shfl_xor_sync(0xffffffffu, acc.w, dl));
-          const int d = n4 % p.head_dim;
-          if (n4 / p.head_dim < p.n_q_heads + p.n_kv_heads) {
-            const size_t a = ((size_t)b * p.q_cap + i) * half + (d < half ? d : d - half);
-            const float4 cs = __ldg(reinterpret_cast<const float4*>(p.rope_cos + a));
-            const float4 sn = __ldg(reinterpret_cast<const float4*>(p.rope_sin + a));
-            const float sg = d < half ? -1.f : 1.f;
-            acc.x = fmaf(sg * o.x, sn.x, acc.x * cs.x);
-            acc.y = fmaf(sg * o.y, sn.y, acc.y * cs.y);
-            acc.z = fmaf(sg * o.z, sn.z, acc.z * cs.z);
-            acc.w = fmaf(sg * o.w, sn.w, acc.w * cs.w);
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+          const int rr = rr0 + 4 * j;
+          if (rr >= red_end) break;   // the same for the whole warp
+          float4 acc = accs[j];
+          const int r = row0 + rr;
+          const int b = r / p.q_cap, i = r % p.q_cap;
+          if (rope) {
+            // this lane's 4 features and their partners' (head_dim / 2 features = head_dim / 8 lanes away) turn together;
+            // rr is the same for the whole warp, so every lane is here for the exchange
+            const int dl = p.head_dim >> 3;
+            const float4 o = make_float4(__shfl_xor_sync(0xffffffffu, acc.x, dl), __shfl_xor_sync(0xffffffffu, acc.y, dl),
+                                         __shfl_xor_sync(0xffffffffu, acc.z, dl), __shfl_xor_sync(0xffffffffu, acc.w, dl));
+            const int d = n4 % p.head_dim;
+            if (n4 / p.head_dim < p.n_q_heads + p.n_kv_heads) {
+              const size_t a = ((size_t)b * p.q_cap + i) * half + (d < half ? d : d - half);
+              const float4 cs = __ldg(reinterpret_cast<const float4*>(p.rope_cos + a));
+              const float4 sn = __ldg(reinterpret_cast<const float4*>(p.rope_sin + a));
+              const float sg = d < half ? -1.f : 1.f;
+              acc.x = fmaf(sg * o.x, sn.x, acc.x * cs.x);
+              acc.y = fmaf(sg * o.y, sn.y, acc.y * cs.y);
+              acc.z = fmaf(sg * o.z, sn.z, acc.z * cs.z);
+              acc.w = fmaf(sg * o.w, sn.w, acc.w * cs.w);
+            }
           }
-        }
-        const __nv_bfloat162 lo = __floats2bfloat162_rn(acc.x, acc.y), hi = __floats2bfloat162_rn(acc.z, acc.w);
-        uint2 pk;
-        pk.x = *reinterpret_cast<const uint32_t*>(&lo);
-        pk.y = *reinterpret_cast<const uint32_t*>(&hi);
-        *reinterpret_cast<uint2*>(dst + (size_t)b * b_stride + (size_t)i * row_stride) = pk;
-        if (stage) {
-          const int pos = stage_row(b, i);
-          if (pos >= 0) *reinterpret_cast<uint2*>(stage + (size_t)b * stage_b_stride + (size_t)pos * p.head_dim) = pk;
+          const __nv_bfloat162 lo = __floats2bfloat162_rn(acc.x, acc.y), hi = __floats2bfloat162_rn(acc.z, acc.w);
+          uint2 pk;
+          pk.x = *reinterpret_cast<const uint32_t*>(&lo);
+          pk.y = *reinterpret_cast<const uint32_t*>(&hi);
+          *reinterpret_cast<uint2*>(dst + (size_t)b * b_stride + (size_t)i * row_stride) = pk;
+          if (stage) {
+            const int pos = stage_row(b, i);
+            if (pos >= 0) *reinterpret_cast<uint2*>(stage + (size_t)b * stage_b_stride + (size_t)pos * p.head_dim) = pk;
+          }
         }
       }
     }
@@ -414,9 +467,14 @@ bool make_proj_plan(const dlm_ctx* ctx, int rows, int n_out, int k_total, bool w
   if (stages > chunks_per_split) stages = chunks_per_split;
   if (stages < 2) return false;
   pl.n_stages = stages;
+  // the shared final reduction parks every partial tile's slice of a block's rows in the stages' memory
+  if (pl.n_split > 1 && (long long)stages * stage < (long long)(pl.rows_pad + pl.n_split) * kTileN * 4) {
+    pl.n_split = 1;
+    pl.k_per_split = k_chunks * kChunkK;
+  }
   pl.smem_bytes = 1024 + stages * stage + aux;
   pl.ws_bytes = pl.n_split > 1 ? (size_t)pl.chunks * pl.tiles * pl.n_split * pl.rows_pad * kTileN * sizeof(float) : 0;
-  return (long long)pl.tiles * pl.chunks <= kDlmMaxSplitUnits;
+  return (long long)pl.tiles * pl.chunks <= kDlmMaxSplitUnits / 2;   // two counters per tile
 }
 
 int launch_proj(dlm_ctx* ctx, const ProjPlan& pl, ProjParams& p, const CUtensorMap& tm_w, const CUtensorMap& tm_x, void* workspace,
