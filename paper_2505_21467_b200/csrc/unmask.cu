@@ -53,7 +53,12 @@ __device__ __forceinline__ void take_better(float& m, int& i, float m2, int i2) 
 // One block reduces chunk blockIdx.x (chunk_len logits) of logit row `row` to a Triple.  Every
 // thread streams its share with U independent 16-byte loads in flight and keeps a running
 // (max, lowest argmax, sum of exp(z - max)); the block combines them with a fixed tree.
-template <int U>
+//
+// kLazy (blocks that make several passes): the loop tracks only the running maximum and the pass in which it last
+// grew, one instruction per logit instead of three (the loop is bound by instruction issue); after the block's
+// maximum is known, the few threads that hold it read their 16-byte vectors of that pass again (L2) and find its first
+// position.  Same maximum, same lowest index, same sum as the eager form.
+template <int U, bool kLazy>
 __device__ __forceinline__ void reduce_chunk(const float* __restrict__ logits, int vocab, int chunk_len, int n_chunks,
                                              Triple* partial, int row) {
   const int chunk = blockIdx.x;
@@ -65,27 +70,37 @@ __device__ __forceinline__ void reduce_chunk(const float* __restrict__ logits, i
 
   float m = -CUDART_INF_F, s = 0.f;
   int mi = 0x7fffffff;
+  int base_of_max = begin;   // kLazy: the pass in which the running maximum last grew
   const bool vec_ok = (((uintptr_t)(z + begin)) & 15) == 0;
-  for (int base = begin; base < end; base += kStep) {
-    float x[U * 4];
-    // thread t owns vectors t, t + 256, ... of the iteration: ascending indices within a thread
+  // thread t owns vectors t, t + 256, ... of a pass: ascending indices within a thread
+  auto load_pass = [&](int base, float (&x)[U * 4], bool streaming) {
 #pragma unroll
     for (int u = 0; u < U; ++u) {
       const int e = base + (u * kThreads + tid) * 4;
       if (vec_ok && e + 3 < end) {
-        const float4 v = __ldcs(reinterpret_cast<const float4*>(z + e));
+        const float4 v = streaming ? __ldcs(reinterpret_cast<const float4*>(z + e)) : __ldcg(reinterpret_cast<const float4*>(z + e));
         x[4 * u + 0] = v.x; x[4 * u + 1] = v.y; x[4 * u + 2] = v.z; x[4 * u + 3] = v.w;
       } else {
 #pragma unroll
         for (int c = 0; c < 4; ++c) x[4 * u + c] = (e + c < end) ? z[e + c] : -CUDART_INF_F;
       }
     }
+  };
+  for (int base = begin; base < end; base += kStep) {
+    float x[U * 4];
+    load_pass(base, x, true);
     float bm = m;
+    if (kLazy) {
 #pragma unroll
-    for (int u = 0; u < U; ++u)
+      for (int u = 0; u < U * 4; ++u) bm = fmaxf(bm, x[u]);   // ignores NaN, as the comparison below does
+      if (bm > m) base_of_max = base;
+    } else {
 #pragma unroll
-      for (int c = 0; c < 4; ++c)
-        if (x[4 * u + c] > bm) { bm = x[4 * u + c]; mi = base + (u * kThreads + tid) * 4 + c; }
+      for (int u = 0; u < U; ++u)
+#pragma unroll
+        for (int c = 0; c < 4; ++c)
+          if (x[4 * u + c] > bm) { bm = x[4 * u + c]; mi = base + (u * kThreads + tid) * 4 + c; }
+    }
     if (bm > m) {   // the running sum follows the running maximum
       s *= __expf(m - bm);
       m = bm;
@@ -97,25 +112,56 @@ __device__ __forceinline__ void reduce_chunk(const float* __restrict__ logits, i
       for (int u = 0; u < U * 4; ++u) s += ex2_ftz((x[u] - m) * 1.4426950408889634f);
     }
   }
-  // block maximum and its lowest index
-  float wm = m;
-  int wi = mi;
-#pragma unroll
-  for (int o = 16; o > 0; o >>= 1) {
-    const float m2 = __shfl_xor_sync(0xffffffffu, wm, o);
-    const int i2 = __shfl_xor_sync(0xffffffffu, wi, o);
-    take_better(wm, wi, m2, i2);
-  }
   __shared__ float sm_m[kThreads / 32];
   __shared__ int sm_i[kThreads / 32];
   __shared__ float sm_s[kThreads / 32];
   const int warp = tid >> 5, lane = tid & 31;
-  if (lane == 0) { sm_m[warp] = wm; sm_i[warp] = wi; }
-  __syncthreads();
-  float bm = sm_m[0];
-  int bi = sm_i[0];
+  float bm;
+  int bi;
+  if (kLazy) {
+    // block maximum first ...
+    float wm = m;
 #pragma unroll
-  for (int w = 1; w < kThreads / 32; ++w) take_better(bm, bi, sm_m[w], sm_i[w]);
+    for (int o = 16; o > 0; o >>= 1) {
+      const float m2 = __shfl_xor_sync(0xffffffffu, wm, o);
+      wm = m2 > wm ? m2 : wm;
+    }
+    if (lane == 0) sm_m[warp] = wm;
+    __syncthreads();
+    bm = sm_m[0];
+#pragma unroll
+    for (int w = 1; w < kThreads / 32; ++w) bm = sm_m[w] > bm ? sm_m[w] : bm;
+    // ... then its lowest index: a thread that holds it finds its first position in the pass where its maximum last grew
+    int wi = 0x7fffffff;
+    if (m == bm && bm > -CUDART_INF_F) {
+      float x[U * 4];
+      load_pass(base_of_max, x, false);
+#pragma unroll
+      for (int u = U - 1; u >= 0; --u)
+#pragma unroll
+        for (int c = 3; c >= 0; --c)
+          if (x[4 * u + c] == bm) wi = base_of_max + (u * kThreads + tid) * 4 + c;
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) wi = min(wi, __shfl_xor_sync(0xffffffffu, wi, o));
+    if (lane == 0) sm_i[warp] = wi;
+  } else {
+    // block maximum and its lowest index
+    float wm = m;
+    int wi = mi;
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+      const float m2 = __shfl_xor_sync(0xffffffffu, wm, o);
+      const int i2 = __shfl_xor_sync(0xffffffffu, wi, o);
+      take_better(wm, wi, m2, i2);
+    }
+    if (lane == 0) { sm_m[warp] = wm; sm_i[warp] = wi; }
+    __syncthreads();
+    bm = sm_m[0];
+    bi = sm_i[0];
+#pragma unroll
+    for (int w = 1; w < kThreads / 32; ++w) take_better(bm, bi, sm_m[w], sm_i[w]);
+  }
   // sums re-based on the block maximum; a thread that saw only -inf contributes nothing
   float t = (m > -CUDART_INF_F) ? s * __expf(m - bm) : 0.f;
 #pragma unroll
@@ -123,6 +169,11 @@ __device__ __forceinline__ void reduce_chunk(const float* __restrict__ logits, i
   if (lane == 0) sm_s[warp] = t;
   __syncthreads();
   if (tid == 0) {
+    if (kLazy) {
+      bi = sm_i[0];
+#pragma unroll
+      for (int w = 1; w < kThreads / 32; ++w) bi = min(bi, sm_i[w]);
+    }
     float total = 0.f;
 #pragma unroll
     for (int w = 0; w < kThreads / 32; ++w) total += sm_s[w];
@@ -240,14 +291,14 @@ __device__ void select_batch(const Triple* partial, int n_chunks, int b, const S
   if (tid == 0) a.n_sel[b] = count;
 }
 
-template <int U>
+template <int U, bool kLazy>
 __global__ void __launch_bounds__(kThreads)
 vocab_reduce_kernel(const float* __restrict__ logits, int vocab, int chunk_len, int n_chunks, Triple* partial,
                     unsigned int* tickets, const SelectArgs sel) {
   dlm_grid_dependency_wait();
   dlm_trigger_dependents();
   const int row = blockIdx.y;
-  if (sel.masked[row]) reduce_chunk<U>(logits, vocab, chunk_len, n_chunks, partial, row);
+  if (sel.masked[row]) reduce_chunk<U, kLazy>(logits, vocab, chunk_len, n_chunks, partial, row);
   if (tickets == nullptr) return;
   // the last block of this batch element to get here runs its selection
   __shared__ bool is_last;
@@ -298,8 +349,10 @@ int launch_unmask(const float* logits, int batch, int block_len, int vocab, uint
   a.sel_idx = sel_idx; a.n_sel = n_sel;
   const dim3 grid(n_chunks, batch * block_len);
   cudaError_t e;
-  if (U == 4) e = dlm_launch(vocab_reduce_kernel<4>, grid, dim3(kThreads), 0, s, logits, vocab, chunk_len, n_chunks, partial, tickets, a);
-  else e = dlm_launch(vocab_reduce_kernel<8>, grid, dim3(kThreads), 0, s, logits, vocab, chunk_len, n_chunks, partial, tickets, a);
+  // blocks of several passes find the argmax's index after the fact (see reduce_chunk)
+  if (U == 4) e = dlm_launch(vocab_reduce_kernel<4, false>, grid, dim3(kThreads), 0, s, logits, vocab, chunk_len, n_chunks, partial, tickets, a);
+  else if (passes < 2) e = dlm_launch(vocab_reduce_kernel<8, false>, grid, dim3(kThreads), 0, s, logits, vocab, chunk_len, n_chunks, partial, tickets, a);
+  else e = dlm_launch(vocab_reduce_kernel<8, true>, grid, dim3(kThreads), 0, s, logits, vocab, chunk_len, n_chunks, partial, tickets, a);
   if (e != cudaSuccess) return -1;
   if (tickets != nullptr) return 1;
   if (dlm_launch(unmask_select_kernel, dim3(batch), dim3(kThreads), 0, s, partial, n_chunks, a) != cudaSuccess) return -1;
