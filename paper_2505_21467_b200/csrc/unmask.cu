@@ -54,10 +54,10 @@ __device__ __forceinline__ void take_better(float& m, int& i, float m2, int i2) 
 // thread streams its share with U independent 16-byte loads in flight and keeps a running
 // (max, lowest argmax, sum of exp(z - max)); the block combines them with a fixed tree.
 //
-// kLazy (blocks that make several passes): the loop tracks only the running maximum and the pass in which it last
-// grew, one instruction per logit instead of three (the loop is bound by instruction issue); after the block's
-// maximum is known, the few threads that hold it read their 16-byte vectors of that pass again (L2) and find its first
-// position.  Same maximum, same lowest index, same sum as the eager form.
+// kLazy (blocks that make several passes): the loop tracks only the running maximum and the half pass in which it
+// last grew, one instruction per logit instead of three; after the block's maximum is known, the few threads that
+// hold it read their 16-byte vectors of that half pass again (L2) and find its first position.  Same maximum and
+// same lowest index as the eager form; the sum is taken half pass by half pass (see the pipeline below).
 template <int U, bool kLazy>
 __device__ __forceinline__ void reduce_chunk(const float* __restrict__ logits, int vocab, int chunk_len, int n_chunks,
                                              Triple* partial, int row) {
@@ -86,30 +86,70 @@ __device__ __forceinline__ void reduce_chunk(const float* __restrict__ logits, i
       }
     }
   };
-  for (int base = begin; base < end; base += kStep) {
-    float x[U * 4];
-    load_pass(base, x, true);
-    float bm = m;
-    if (kLazy) {
+  int half_of_max = 0;       // kLazy: ... and the half of that pass
+  // one half of a pass: vectors u in [h U/2, (h + 1) U/2) of this thread
+  auto load_half = [&](int base, int h, float (&x)[U * 2], bool streaming) {
 #pragma unroll
-      for (int u = 0; u < U * 4; ++u) bm = fmaxf(bm, x[u]);   // ignores NaN, as the comparison below does
-      if (bm > m) base_of_max = base;
-    } else {
+    for (int u = 0; u < U / 2; ++u) {
+      const int e = base + ((h * (U / 2) + u) * kThreads + tid) * 4;
+      if (vec_ok && e + 3 < end) {
+        const float4 v = streaming ? __ldcs(reinterpret_cast<const float4*>(z + e)) : __ldcg(reinterpret_cast<const float4*>(z + e));
+        x[4 * u + 0] = v.x; x[4 * u + 1] = v.y; x[4 * u + 2] = v.z; x[4 * u + 3] = v.w;
+      } else {
+#pragma unroll
+        for (int c = 0; c < 4; ++c) x[4 * u + c] = (e + c < end) ? z[e + c] : -CUDART_INF_F;
+      }
+    }
+  };
+  if (kLazy) {
+    // Software pipeline over half passes: while one half's arithmetic runs, the other half's loads (of this pass or
+    // the next) are in flight, so a thread always has U/2 to U vectors outstanding.  With whole passes a thread had
+    // nothing in flight during its arithmetic, about 40 % of the time.
+    float xa[U * 2], xb[U * 2];
+    auto process = [&](const float (&x)[U * 2], int base, int h) {
+      float bm = m;
+#pragma unroll
+      for (int u = 0; u < U * 2; ++u) bm = fmaxf(bm, x[u]);   // ignores NaN, as a comparison would
+      if (bm > m) {   // the running sum follows the running maximum
+        base_of_max = base;
+        half_of_max = h;
+        s *= __expf(m - bm);
+        m = bm;
+      }
+      if (m > -CUDART_INF_F) {
+#pragma unroll
+        for (int u = 0; u < U * 2; ++u) s += ex2_ftz((x[u] - m) * 1.4426950408889634f);
+      }
+    };
+    load_half(begin, 0, xa, true);
+    load_half(begin, 1, xb, true);
+    for (int base = begin; base < end; base += kStep) {
+      const bool more = base + kStep < end;
+      process(xa, base, 0);
+      if (more) load_half(base + kStep, 0, xa, true);
+      process(xb, base, 1);
+      if (more) load_half(base + kStep, 1, xb, true);
+    }
+  } else {
+    for (int base = begin; base < end; base += kStep) {
+      float x[U * 4];
+      load_pass(base, x, true);
+      float bm = m;
 #pragma unroll
       for (int u = 0; u < U; ++u)
 #pragma unroll
         for (int c = 0; c < 4; ++c)
           if (x[4 * u + c] > bm) { bm = x[4 * u + c]; mi = base + (u * kThreads + tid) * 4 + c; }
-    }
-    if (bm > m) {   // the running sum follows the running maximum
-      s *= __expf(m - bm);
-      m = bm;
-    }
-    if (m > -CUDART_INF_F) {
-      // exp(x - m) as 2^((x - m) log2(e)) with the flush-to-zero SFU instruction: the library exponential spends
-      // three more instructions per logit on denormal results, and the loop is bound by instruction issue
+      if (bm > m) {   // the running sum follows the running maximum
+        s *= __expf(m - bm);
+        m = bm;
+      }
+      if (m > -CUDART_INF_F) {
+        // exp(x - m) as 2^((x - m) log2(e)) with the flush-to-zero SFU instruction: the library exponential spends
+        // three more instructions per logit on denormal results, and the loop is bound by instruction issue
 #pragma unroll
-      for (int u = 0; u < U * 4; ++u) s += ex2_ftz((x[u] - m) * 1.4426950408889634f);
+        for (int u = 0; u < U * 4; ++u) s += ex2_ftz((x[u] - m) * 1.4426950408889634f);
+      }
     }
   }
   __shared__ float sm_m[kThreads / 32];
@@ -134,13 +174,13 @@ __device__ __forceinline__ void reduce_chunk(const float* __restrict__ logits, i
     // ... then its lowest index: a thread that holds it finds its first position in the pass where its maximum last grew
     int wi = 0x7fffffff;
     if (m == bm && bm > -CUDART_INF_F) {
-      float x[U * 4];
-      load_pass(base_of_max, x, false);
+      float x[U * 2];
+      load_half(base_of_max, half_of_max, x, false);
 #pragma unroll
-      for (int u = U - 1; u >= 0; --u)
+      for (int u = U / 2 - 1; u >= 0; --u)
 #pragma unroll
         for (int c = 3; c >= 0; --c)
-          if (x[4 * u + c] == bm) wi = base_of_max + (u * kThreads + tid) * 4 + c;
+          if (x[4 * u + c] == bm) wi = base_of_max + ((half_of_max * (U / 2) + u) * kThreads + tid) * 4 + c;
     }
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) wi = min(wi, __shfl_xor_sync(0xffffffffu, wi, o));
